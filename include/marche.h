@@ -1,0 +1,257 @@
+/*
+ * marche.h - C ABI of libmarche: the per-decoding-step hot path of MARche
+ * (cache-aware attention with selective KV refresh for masked autoregressive
+ * image generation) on one NVIDIA B200 (sm_100a).
+ *
+ * Conventions that hold for every call unless a call says otherwise
+ * -----------------------------------------------------------------
+ * Pointers   "device" pointers address global memory of the GPU that was current
+ *            when marche_create() ran; "host" pointers address ordinary host
+ *            memory.  The library never allocates or frees device memory: the
+ *            caller owns hidden states, the K/V cache, index arrays, weights
+ *            and the workspace, and keeps them alive until the stream has
+ *            finished the call.  The library owns only the small host-side
+ *            marche_ctx.
+ * Streams    `stream` is a cudaStream_t passed as an opaque pointer (NULL = the
+ *            default stream).  All device work is enqueued on it and the call
+ *            returns without waiting for it (asynchronous), except where noted.
+ * Notation   B batch rows, S tokens per sample, D width = H heads x dh,
+ *            F MLP width, L blocks, nA active tokens per sample, nG generating
+ *            ("new") tokens per sample, M = B*nA rows.  `T` is the compute
+ *            type selected by marche_config.dtype (float or bf16).
+ * Index sets int32, device, row-major [B][n] with the same n for every sample;
+ *            entries are token positions in [0, S), unique within a sample.
+ * Layouts    hidden / hidden_out  float [B][S][D]
+ *            K/V cache            T [L][2][B][S][D]; [l][0] holds K, [l][1] V;
+ *                                 head h occupies columns h*dh .. (h+1)*dh-1
+ *            weight matrices      T [out][in] row-major; LayerNorm parameters
+ *                                 and all biases are float
+ * Errors     0 (MARCHE_OK) on success, a negative MARCHE_E* code otherwise; no
+ *            C++ exception crosses the boundary and no device code traps.  When
+ *            a code other than MARCHE_OK is returned because of argument
+ *            checking, nothing was enqueued.  CUDA launch errors are reported
+ *            as MARCHE_ECUDA (text via marche_last_error()).  Index contents
+ *            are not validated on the device (out-of-range or duplicate
+ *            entries are undefined behaviour) unless the call says so.
+ * Threads    a marche_ctx may be used from one host thread at a time.
+ */
+#ifndef MARCHE_H_
+#define MARCHE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct marche_ctx marche_ctx;
+typedef void* marche_stream; /* cudaStream_t */
+
+enum { MARCHE_F32 = 0, MARCHE_BF16 = 1 };
+
+enum {
+  MARCHE_OK = 0,
+  MARCHE_EINVAL = -1,     /* NULL pointer, negative size, inconsistent arguments          */
+  MARCHE_ESHAPE = -2,     /* dimensions this build has no kernel for                      */
+  MARCHE_EWORKSPACE = -3, /* workspace (or cache buffer) smaller than required            */
+  MARCHE_ECACHE = -4,     /* cache-aware step on a cache no full step has filled          */
+  MARCHE_EINDEX = -5,     /* marche_validate_indices found a bad index set                */
+  MARCHE_ECUDA = -6,      /* a CUDA runtime / driver call failed                          */
+  MARCHE_ETIMEOUT = -7    /* a bounded device-side wait gave up (see marche_device_status)*/
+};
+
+/* Epilogues of marche_linear. */
+enum {
+  MARCHE_EPI_BIAS = 0,          /* out T[M][N]      = acc + bias                          */
+  MARCHE_EPI_BIAS_RESIDUAL = 1, /* out float[M][N] += acc + bias   (read-modify-write)    */
+  MARCHE_EPI_BIAS_GELU = 2      /* out T[M][N]      = GELU_erf(acc + bias)                */
+};
+
+typedef struct {
+  int32_t n_blocks;     /* L                                                              */
+  int32_t n_enc_blocks; /* E; only used for the default score layer                       */
+  int32_t width;        /* D, multiple of 128, <= 2048                                    */
+  int32_t n_heads;      /* H                                                              */
+  int32_t head_dim;     /* dh = D / H; 64 or 80 for bf16, any multiple of 16 <= 128 f32   */
+  int32_t mlp_dim;      /* F, multiple of 128                                             */
+  int32_t seq_len;      /* S = image tokens + buffer tokens, <= 2048                      */
+  int32_t n_buffer;     /* informational (buffer tokens are ordinary tokens here)         */
+  int32_t batch;        /* B, already doubled for classifier-free guidance                */
+  int32_t dtype;        /* MARCHE_F32 or MARCHE_BF16: GEMM/attention operands and cache   */
+  int32_t score_layer;  /* 0-based block whose attention yields the relevance scores;
+                           -1 selects the second decoder block, E+1 (Section 4.2)         */
+  float ln_eps;         /* LayerNorm epsilon; <= 0 selects 1e-6                           */
+} marche_config;
+
+/* One entry per block; all device pointers.  The block is the standard pre-LN
+ * transformer block that Algorithm 1 abbreviates:  x += Wo*Attn(LN1(x)) + bo;
+ * x += W2*GELU(W1*LN2(x) + b1) + b2.  w_qkv is [3D][D] with rows ordered q, k, v. */
+typedef struct {
+  const float* ln1_g; const float* ln1_b;
+  const void* w_qkv;  const float* b_qkv;
+  const void* w_o;    const float* b_o;
+  const float* ln2_g; const float* ln2_b;
+  const void* w_fc1;  const float* b_fc1;
+  const void* w_fc2;  const float* b_fc2;
+} marche_block_weights;
+
+/* ---------------------------------------------------------------- life cycle */
+
+/* Creates the host-side context for one model shape on the current device.
+ * `blocks` is a host array of cfg->n_blocks structs (copied).  Synchronous; no
+ * device memory is allocated.  MARCHE_ESHAPE for unsupported dimensions. */
+int marche_create(const marche_config* cfg, const marche_block_weights* blocks, marche_ctx** out);
+void marche_destroy(marche_ctx* ctx);
+
+/* Bytes of the K/V cache, L*2*B*S*D*sizeof(T), and of the scratch workspace a
+ * step with up to `max_active` active tokens per sample needs (S for a full
+ * step).  The workspace must be 256-byte aligned. */
+size_t marche_cache_bytes(const marche_ctx* ctx);
+size_t marche_workspace_bytes(const marche_ctx* ctx, int max_active);
+
+/* Zero-fills `kv_cache` (device) and records it as "not filled": a cache-aware
+ * step on it fails with MARCHE_ECACHE until a full step has run on it (the
+ * initial full refresh of Section 4.3). */
+int marche_init_cache(marche_ctx* ctx, void* kv_cache, size_t bytes, marche_stream stream);
+
+/* ---------------------------------------------------------------- the step */
+
+/* One cache-aware decoding step: Algorithm 1 lines 4-11 for every block, with
+ * the relevance scores of Section 4.2 taken at block `score_layer` and the
+ * top-K refresh selection applied to them (the selection feeds the NEXT step).
+ *
+ *   hidden       in   device float [B][S][D]  stack input (token embeddings)
+ *   kv_cache     i/o  device T [L][2][B][S][D]; rows active_idx of every block
+ *                     are overwritten with fresh K, V, all other rows keep their
+ *                     bytes
+ *   active_idx   in   device int32 [B][n_active]   A = G u N u R
+ *   new_idx      in   device int32 [B][n_new]      G, a subset of active_idx; the
+ *                     queries of these tokens produce the relevance scores
+ *   exclude_idx  in   device int32 [B][n_excl] or NULL: tokens that must not be
+ *                     selected besides new_idx (the caller passes the tokens
+ *                     the next step generates); disjoint from new_idx
+ *   refresh_ratio     K = min(S - n_new - n_excl, floor(ratio*S + 1/2))
+ *   hidden_out   out  device float [B][S][D]; rows active_idx receive the stack
+ *                     output, other rows keep their bytes.  May not alias hidden.
+ *   refresh_idx  out  device int32 [B][K], ascending token index per sample; K
+ *                     highest scores, ties broken towards the lower index.  Must
+ *                     hold B*floor(ratio*S+1/2) entries.  May be NULL: no selection.
+ *   n_refresh    out  host int, receives K (may be NULL)
+ *   workspace         device scratch of marche_workspace_bytes(ctx, n_active)
+ * Errors: MARCHE_ECACHE if kv_cache was never filled by marche_full_step;
+ * MARCHE_EINVAL for n_active < 1 or > S, n_new > n_active, NULL buffers;
+ * MARCHE_EWORKSPACE. */
+int marche_step(marche_ctx* ctx, const float* hidden, void* kv_cache,
+                const int32_t* active_idx, int n_active,
+                const int32_t* new_idx, int n_new,
+                const int32_t* exclude_idx, int n_excl,
+                float refresh_ratio, float* hidden_out,
+                int32_t* refresh_idx, int* n_refresh,
+                void* workspace, size_t workspace_bytes, marche_stream stream);
+
+/* The same stack with every token active (active_idx = 0..S-1): the initial
+ * full refresh that fills the cache (Section 4.3) and the full-recompute MAR
+ * baseline (Section 3, Motivation).  Marks kv_cache as filled.  Workspace of
+ * marche_workspace_bytes(ctx, S). */
+int marche_full_step(marche_ctx* ctx, const float* hidden, void* kv_cache,
+                     const int32_t* new_idx, int n_new,
+                     const int32_t* exclude_idx, int n_excl,
+                     float refresh_ratio, float* hidden_out,
+                     int32_t* refresh_idx, int* n_refresh,
+                     void* workspace, size_t workspace_bytes, marche_stream stream);
+
+/* Top-K refresh selection alone (Section 4.2, "select the top-K tokens with the
+ * highest relevance scores"): scores device float [B][S] (finite); candidates
+ * are all tokens outside new_idx and exclude_idx; writes refresh_idx device
+ * int32 [B][k] ascending; order (score descending, index ascending); -0 == +0.
+ * `mask_scratch` is device scratch of B*S bytes.  MARCHE_EINVAL if
+ * k > S - n_new - n_excl or k < 0; k == 0 enqueues nothing. */
+int marche_select_refresh(marche_ctx* ctx, const float* scores,
+                          const int32_t* new_idx, int n_new,
+                          const int32_t* exclude_idx, int n_excl,
+                          int k, int32_t* refresh_idx, void* mask_scratch, marche_stream stream);
+
+/* Copies the relevance scores float [B][S] that the last step left in
+ * `workspace` to `scores_out` (device).  Section 4.2: attention probability
+ * from the generating tokens to each token, summed over heads and queries. */
+int marche_get_scores(marche_ctx* ctx, const void* workspace, float* scores_out, marche_stream stream);
+
+/* Algorithm 1 line 4, A = G u N u R, built on the device so that a generation
+ * loop needs no host round trip: active_idx[b] = new_idx[b] | prev_idx[b] |
+ * refresh_idx[b] (concatenation; the caller guarantees disjointness).  Any of
+ * the three may have n = 0 (pointer then ignored).  active_idx device int32
+ * [B][n_new + n_prev + n_refresh]. */
+int marche_build_active(marche_ctx* ctx, const int32_t* new_idx, int n_new,
+                        const int32_t* prev_idx, int n_prev,
+                        const int32_t* refresh_idx, int n_refresh,
+                        int32_t* active_idx, marche_stream stream);
+
+/* Row scatter dst[b][idx[b][j]][:] = rows[b][j][:] for float [B][n][D] rows into
+ * float [B][S][D]; the step uses it for hidden_out (only active rows are
+ * written, cf. Algorithm 1 line 9) and a generation driver uses it to insert the
+ * tokens sampled after a step (Eq. 3-4) into the stack input. */
+int marche_scatter_rows(marche_ctx* ctx, const float* rows, const int32_t* idx, int n,
+                        float* dst, marche_stream stream);
+
+/* Checks index sets on the device (range, uniqueness within a sample, new_idx a
+ * subset of active_idx, exclude_idx disjoint from new_idx) and waits for the
+ * result: MARCHE_OK or MARCHE_EINDEX.  Synchronous.  active_idx may be NULL
+ * (n_active = 0) to skip its checks. */
+int marche_validate_indices(marche_ctx* ctx, const int32_t* active_idx, int n_active,
+                            const int32_t* new_idx, int n_new,
+                            const int32_t* exclude_idx, int n_excl, marche_stream stream);
+
+/* ---------------------------------------------------------------- single kernels
+ * The step is a fixed sequence of the calls below; they are exported so that
+ * each kernel can be checked and measured on its own. */
+
+/* Gather + LayerNorm (Algorithm 1 line 5, input side): for r = b*n + j,
+ *   x = src[b][idx ? idx[b][j] : j][:]   (src float [B][src_rows][D])
+ *   x_out[r][:] = x                      (float [B*n][D], skipped when NULL)
+ *   u_out[r][:] = (x-mean)/sqrt(var+eps)*gamma + beta   (T [B*n][D])
+ * Statistics in fp32 from the row held in registers (two passes). */
+int marche_gather_layernorm(marche_ctx* ctx, const float* src, int src_rows, const int32_t* idx, int n,
+                            const float* gamma, const float* beta, float* x_out, void* u_out,
+                            marche_stream stream);
+
+/* out = epilogue(a * w^T + bias): a T [M][K] with row stride lda elements,
+ * w T [N][K], bias float [N], out [M][N] dense (type per epilogue).  The QKV,
+ * output and MLP projections on active rows only (Algorithm 1 lines 5 and 9).
+ * bf16: K % 64 == 0, N % 128 == 0, lda % 8 == 0.  fp32 accumulation. */
+int marche_linear(marche_ctx* ctx, const void* a, int lda, int M, const void* w, const float* bias,
+                  int N, int K, int epilogue, void* out, marche_stream stream);
+
+/* Cache write-back (Algorithm 1 line 11): for r = b*n + j,
+ *   cache_layer[0][b][idx[b][j]][:] = k[r][:], cache_layer[1][b][..] = v[r][:]
+ * k, v T [B*n][D] with row stride ld_kv elements; cache_layer = T [2][B][S][D]
+ * (one block's slice of the cache); idx NULL means the identity (n == S). */
+int marche_scatter_kv(marche_ctx* ctx, const void* k, const void* v, int ld_kv,
+                      const int32_t* idx, int n, void* cache_layer, marche_stream stream);
+
+/* Attention of the active queries over ALL S cached rows of one block, unmasked
+ * (Algorithm 1 lines 6-8, equal to Eq. 5 by Appendix A once the fresh K, V of
+ * the active rows are in the cache), with the fused relevance reduction of
+ * Section 4.2:
+ *   q T [B*n][D] with row stride ld_q; o T [B*n][D] dense;
+ *   is_new  device uint8 [B][n] flags of the scoring queries, or NULL: no scores;
+ *   score_partial device float [B][H][S]: per head, sum over flagged queries of
+ *   the softmax weights (overwritten, not accumulated); ignored when is_new NULL. */
+int marche_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void* cache_layer,
+                     const uint8_t* is_new, float* score_partial, void* o, marche_stream stream);
+
+/* ---------------------------------------------------------------- diagnostics */
+const char* marche_strerror(int code);
+/* Text of the last CUDA error this context saw ("" if none). */
+const char* marche_last_error(const marche_ctx* ctx);
+/* Status word that bounded waits inside the kernels set when they give up
+ * (0 = none; otherwise a kernel-specific code, and the step's results are
+ * invalid).  It lives in pinned host memory owned by the context; synchronise
+ * the stream before reading it. */
+int marche_device_status(const marche_ctx* ctx);
+void marche_clear_device_status(marche_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MARCHE_H_ */

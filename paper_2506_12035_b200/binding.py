@@ -1,0 +1,247 @@
+"""ctypes binding of libmarche.so: one Python method per C-ABI entry point.
+
+Argument marshalling only - every step of the hot path runs inside the
+library's CUDA kernels.  PyTorch tensors provide device memory and streams.
+There is no fallback: if the shared library is missing or a call fails, an
+exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmarche.so")
+
+MARCHE_F32, MARCHE_BF16 = 0, 1
+EPI_BIAS, EPI_BIAS_RESIDUAL, EPI_BIAS_GELU = 0, 1, 2
+ERRORS = {-1: "EINVAL", -2: "ESHAPE", -3: "EWORKSPACE", -4: "ECACHE", -5: "EINDEX", -6: "ECUDA", -7: "ETIMEOUT"}
+
+BLOCK_FIELDS = ("ln1_g", "ln1_b", "w_qkv", "b_qkv", "w_o", "b_o",
+                "ln2_g", "ln2_b", "w_fc1", "b_fc1", "w_fc2", "b_fc2")
+MATRIX_FIELDS = ("w_qkv", "w_o", "w_fc1", "w_fc2")
+
+
+class MarcheConfig(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_blocks", "n_enc_blocks", "width", "n_heads", "head_dim", "mlp_dim",
+                                         "seq_len", "n_buffer", "batch", "dtype", "score_layer")] + [("ln_eps", C.c_float)]
+
+
+class MarcheBlockWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in BLOCK_FIELDS]
+
+
+class MarcheError(RuntimeError):
+    def __init__(self, code: int, detail: str = ""):
+        self.code = code
+        super().__init__("libmarche: %s (%d) %s" % (ERRORS.get(code, "?"), code, detail))
+
+
+_vp, _i, _f, _sz = C.c_void_p, C.c_int, C.c_float, C.c_size_t
+_SIGNATURES = {
+    "marche_create": (C.c_int, [C.POINTER(MarcheConfig), C.POINTER(MarcheBlockWeights), C.POINTER(_vp)]),
+    "marche_destroy": (None, [_vp]),
+    "marche_cache_bytes": (_sz, [_vp]),
+    "marche_workspace_bytes": (_sz, [_vp, _i]),
+    "marche_init_cache": (C.c_int, [_vp, _vp, _sz, _vp]),
+    "marche_step": (C.c_int, [_vp, _vp, _vp, _vp, _i, _vp, _i, _vp, _i, _f, _vp, _vp, C.POINTER(C.c_int), _vp, _sz, _vp]),
+    "marche_full_step": (C.c_int, [_vp, _vp, _vp, _vp, _i, _vp, _i, _f, _vp, _vp, C.POINTER(C.c_int), _vp, _sz, _vp]),
+    "marche_select_refresh": (C.c_int, [_vp, _vp, _vp, _i, _vp, _i, _i, _vp, _vp, _vp]),
+    "marche_get_scores": (C.c_int, [_vp, _vp, _vp, _vp]),
+    "marche_build_active": (C.c_int, [_vp, _vp, _i, _vp, _i, _vp, _i, _vp, _vp]),
+    "marche_scatter_rows": (C.c_int, [_vp, _vp, _vp, _i, _vp, _vp]),
+    "marche_validate_indices": (C.c_int, [_vp, _vp, _i, _vp, _i, _vp, _i, _vp]),
+    "marche_gather_layernorm": (C.c_int, [_vp, _vp, _i, _vp, _i, _vp, _vp, _vp, _vp, _vp]),
+    "marche_linear": (C.c_int, [_vp, _vp, _i, _i, _vp, _vp, _i, _i, _i, _vp, _vp]),
+    "marche_scatter_kv": (C.c_int, [_vp, _vp, _vp, _i, _vp, _i, _vp, _vp]),
+    "marche_attention": (C.c_int, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
+    "marche_strerror": (C.c_char_p, [C.c_int]),
+    "marche_last_error": (C.c_char_p, [_vp]),
+    "marche_device_status": (C.c_int, [_vp]),
+    "marche_clear_device_status": (None, [_vp]),
+}
+EXPORTED_SYMBOLS = tuple(_SIGNATURES)
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Loads libmarche.so (built in-tree by paper_2506_12035_b200.build); raises if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                "%s not found: build it with `python -m paper_2506_12035_b200.build` (no fallback exists)" % LIB_PATH)
+        lib = C.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device-resident contiguous tensor required"
+    return t.data_ptr()
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> Optional[int]:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream or None
+
+
+def upload_weights(blocks: Sequence[Dict], dtype: str, device="cuda") -> List[Dict[str, torch.Tensor]]:
+    """Copies per-block parameter arrays (NumPy or torch, fp32) to the device: the four
+    matrices in the compute type, LayerNorm parameters and biases in fp32."""
+    mt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    out = []
+    for blk in blocks:
+        d = {}
+        for name in BLOCK_FIELDS:
+            t = torch.as_tensor(blk[name])
+            d[name] = t.to(device=device, dtype=mt if name in MATRIX_FIELDS else torch.float32).contiguous()
+        out.append(d)
+    return out
+
+
+class Marche:
+    """One model shape on the current CUDA device.  Methods carry the names of the C
+    calls without the `marche_` prefix and take torch CUDA tensors."""
+
+    def __init__(self, *, L: int, E: int, D: int, H: int, F: int, S: int, B: int, dtype: str,
+                 weights: Sequence[Dict[str, torch.Tensor]], n_buffer: int = 0, score_layer: int = -1,
+                 ln_eps: float = 1e-6):
+        if not torch.cuda.is_available():
+            raise RuntimeError("libmarche needs a CUDA device; there is no CPU path")
+        self.lib = load_library()
+        self.L, self.E, self.D, self.H, self.F, self.S, self.B = L, E, D, H, F, S, B
+        self.dtype = dtype
+        self.torch_dtype = torch.bfloat16 if dtype == "bf16" else torch.float32
+        self.weights = list(weights)          # keeps the device tensors alive
+        assert len(self.weights) == L
+        cfg = MarcheConfig(L, E, D, H, D // H, F, S, n_buffer, B, MARCHE_BF16 if dtype == "bf16" else MARCHE_F32,
+                           score_layer, ln_eps)
+        arr = (MarcheBlockWeights * L)()
+        for l, blk in enumerate(self.weights):
+            for name in BLOCK_FIELDS:
+                t = blk[name]
+                want = self.torch_dtype if name in MATRIX_FIELDS else torch.float32
+                assert t.is_cuda and t.is_contiguous() and t.dtype == want, name
+                setattr(arr[l], name, t.data_ptr())
+        h = C.c_void_p()
+        self._check(self.lib.marche_create(C.byref(cfg), arr, C.byref(h)), None)
+        self.h = h
+
+    @classmethod
+    def from_config(cls, cfg, weights, **kw) -> "Marche":
+        """cfg: any object with attributes L, E, D, H, F, S, B, n_buffer, dtype, ln_eps."""
+        return cls(L=cfg.L, E=cfg.E, D=cfg.D, H=cfg.H, F=cfg.F, S=cfg.S, B=cfg.B, dtype=cfg.dtype, weights=weights,
+                   n_buffer=cfg.n_buffer, ln_eps=cfg.ln_eps, **kw)
+
+    def __del__(self):
+        h = getattr(self, "h", None)
+        if h:
+            self.lib.marche_destroy(h)
+            self.h = None
+
+    def _check(self, rc: int, h="self"):
+        if rc != 0:
+            detail = ""
+            if h == "self" and rc == -6:
+                detail = self.lib.marche_last_error(self.h).decode()
+            raise MarcheError(rc, detail)
+
+    # ------------------------------------------------------------- sizes and buffers
+    def cache_bytes(self) -> int:
+        return self.lib.marche_cache_bytes(self.h)
+
+    def workspace_bytes(self, max_active: int) -> int:
+        return self.lib.marche_workspace_bytes(self.h, max_active)
+
+    def alloc_cache(self) -> torch.Tensor:
+        return torch.empty(self.L, 2, self.B, self.S, self.D, dtype=self.torch_dtype, device="cuda")
+
+    def alloc_workspace(self, max_active: int) -> torch.Tensor:
+        return torch.empty(self.workspace_bytes(max_active), dtype=torch.uint8, device="cuda")
+
+    # ------------------------------------------------------------- C calls
+    def init_cache(self, kv_cache, stream=None):
+        self._check(self.lib.marche_init_cache(self.h, _ptr(kv_cache), kv_cache.numel() * kv_cache.element_size(),
+                                               _stream(stream)))
+
+    def step(self, hidden, kv_cache, active_idx, new_idx, exclude_idx, refresh_ratio, hidden_out, refresh_idx,
+             workspace, stream=None) -> int:
+        k = C.c_int(0)
+        self._check(self.lib.marche_step(
+            self.h, _ptr(hidden), _ptr(kv_cache), _ptr(active_idx), active_idx.shape[1],
+            _ptr(new_idx), 0 if new_idx is None else new_idx.shape[1],
+            _ptr(exclude_idx), 0 if exclude_idx is None else exclude_idx.shape[1],
+            refresh_ratio, _ptr(hidden_out), _ptr(refresh_idx), C.byref(k), _ptr(workspace), workspace.numel(),
+            _stream(stream)))
+        return k.value
+
+    def full_step(self, hidden, kv_cache, new_idx, exclude_idx, refresh_ratio, hidden_out, refresh_idx, workspace,
+                  stream=None) -> int:
+        k = C.c_int(0)
+        self._check(self.lib.marche_full_step(
+            self.h, _ptr(hidden), _ptr(kv_cache),
+            _ptr(new_idx), 0 if new_idx is None else new_idx.shape[1],
+            _ptr(exclude_idx), 0 if exclude_idx is None else exclude_idx.shape[1],
+            refresh_ratio, _ptr(hidden_out), _ptr(refresh_idx), C.byref(k), _ptr(workspace), workspace.numel(),
+            _stream(stream)))
+        return k.value
+
+    def select_refresh(self, scores, new_idx, exclude_idx, k, refresh_idx, mask_scratch, stream=None):
+        self._check(self.lib.marche_select_refresh(
+            self.h, _ptr(scores), _ptr(new_idx), 0 if new_idx is None else new_idx.shape[1],
+            _ptr(exclude_idx), 0 if exclude_idx is None else exclude_idx.shape[1], k, _ptr(refresh_idx),
+            _ptr(mask_scratch), _stream(stream)))
+
+    def get_scores(self, workspace, scores_out, stream=None):
+        self._check(self.lib.marche_get_scores(self.h, _ptr(workspace), _ptr(scores_out), _stream(stream)))
+
+    def build_active(self, new_idx, prev_idx, refresh_idx, n_refresh, active_idx, stream=None):
+        self._check(self.lib.marche_build_active(
+            self.h, _ptr(new_idx), 0 if new_idx is None else new_idx.shape[1],
+            _ptr(prev_idx), 0 if prev_idx is None else prev_idx.shape[1],
+            _ptr(refresh_idx) if n_refresh else None, n_refresh, _ptr(active_idx), _stream(stream)))
+
+    def scatter_rows(self, rows, idx, dst, stream=None):
+        self._check(self.lib.marche_scatter_rows(self.h, _ptr(rows), _ptr(idx), idx.shape[1], _ptr(dst),
+                                                 _stream(stream)))
+
+    def validate_indices(self, active_idx, new_idx, exclude_idx, stream=None):
+        self._check(self.lib.marche_validate_indices(
+            self.h, _ptr(active_idx), 0 if active_idx is None else active_idx.shape[1],
+            _ptr(new_idx), 0 if new_idx is None else new_idx.shape[1],
+            _ptr(exclude_idx), 0 if exclude_idx is None else exclude_idx.shape[1], _stream(stream)))
+
+    def gather_layernorm(self, src, idx, n, gamma, beta, x_out, u_out, stream=None):
+        self._check(self.lib.marche_gather_layernorm(self.h, _ptr(src), src.shape[1], _ptr(idx), n, _ptr(gamma),
+                                                     _ptr(beta), _ptr(x_out), _ptr(u_out), _stream(stream)))
+
+    def linear(self, a, w, bias, epilogue, out, M=None, lda=None, stream=None):
+        N, K = w.shape
+        M = a.shape[0] if M is None else M
+        lda = a.stride(0) if lda is None else lda
+        self._check(self.lib.marche_linear(self.h, a.data_ptr(), lda, M, _ptr(w), _ptr(bias), N, K, epilogue,
+                                           _ptr(out), _stream(stream)))
+
+    def scatter_kv(self, k, v, ld_kv, idx, n, cache_layer, stream=None):
+        self._check(self.lib.marche_scatter_kv(self.h, k.data_ptr(), v.data_ptr(), ld_kv, _ptr(idx), n,
+                                               _ptr(cache_layer), _stream(stream)))
+
+    def attention(self, q, ld_q, n, cache_layer, is_new, score_partial, o, stream=None):
+        self._check(self.lib.marche_attention(self.h, q.data_ptr(), ld_q, n, _ptr(cache_layer), _ptr(is_new),
+                                              _ptr(score_partial), _ptr(o), _stream(stream)))
+
+    def device_status(self) -> int:
+        return self.lib.marche_device_status(self.h)
+
+    def clear_device_status(self):
+        self.lib.marche_clear_device_status(self.h)

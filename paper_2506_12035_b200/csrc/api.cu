@@ -1,0 +1,376 @@
+// C ABI of libmarche (see include/marche.h) and the per-step kernel sequence.
+//
+// The step is a fixed chain of launches on the caller's stream, per block:
+//   K1 LayerNorm (with the row gather at block 0) -> K2 QKV projection -> K5 K/V
+//   write-back -> K3 attention over the whole cache (+ score partials at the scoring
+//   block) -> K2 output projection (+residual) -> K1 LayerNorm -> K2 fc1 (+GELU) ->
+//   K2 fc2 (+residual);
+// then once per step the fp32 row scatter into hidden_out and K4 (score reduction +
+// top-K).  Nothing here allocates device memory or synchronises, except where the
+// header says a call is synchronous.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <string>
+#include <utility>
+#include <vector>
+
+#include "../../include/marche.h"
+#include "kernels.h"
+
+using namespace marche;
+
+struct marche_ctx {
+  marche_config cfg;
+  std::vector<marche_block_weights> blocks;
+  int device = 0;
+  bool bf16 = false;
+  size_t eb = 4;
+  float eps = 1e-6f;
+  int score_layer = 0;
+  bool force_simt = false;
+  std::vector<std::pair<const void*, bool>> caches;  // (cache pointer, filled)
+  int* status_host = nullptr;                         // pinned, mapped
+  int* status_dev = nullptr;
+  std::string last_error;
+};
+
+namespace {
+
+inline size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+struct WsLayout {
+  size_t scores, partial, cand, is_new, x, u, qkv, o, g, total;
+};
+
+WsLayout ws_layout(const marche_ctx* c, int nA) {
+  const size_t B = c->cfg.batch, S = c->cfg.seq_len, D = c->cfg.width, F = c->cfg.mlp_dim, H = c->cfg.n_heads;
+  const size_t M = B * (size_t)nA, eb = c->eb;
+  WsLayout w;
+  size_t off = 0;
+  w.scores = off;  off += align256(B * S * sizeof(float));
+  w.partial = off; off += align256(B * H * S * sizeof(float));
+  w.cand = off;    off += align256(B * S);
+  w.is_new = off;  off += align256(M);
+  w.x = off;       off += align256(M * D * sizeof(float));
+  w.u = off;       off += align256(M * D * eb);
+  w.qkv = off;     off += align256(M * 3 * D * eb);
+  w.o = off;       off += align256(M * D * eb);
+  w.g = off;       off += align256(M * F * eb);
+  w.total = off;
+  return w;
+}
+
+int cuda_fail(marche_ctx* c, cudaError_t e, const char* what) {
+  if (c) c->last_error = std::string(what) + ": " + cudaGetErrorString(e);
+  return MARCHE_ECUDA;
+}
+
+#define MARCHE_TRY(call, what)                              \
+  do {                                                      \
+    cudaError_t e__ = (call);                               \
+    if (e__ != cudaSuccess) return cuda_fail(ctx, e__, what); \
+  } while (0)
+
+int refresh_count(float ratio, int S, int n_cand) {
+  const int want = (int)std::floor((double)ratio * (double)S + 0.5);
+  return want < n_cand ? (want < 0 ? 0 : want) : n_cand;
+}
+
+int do_linear(marche_ctx* ctx, const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
+              int epi, void* out, cudaStream_t st) {
+  MARCHE_TRY(launch_gemm_simt(ctx->bf16, a, lda, M, w, bias, N, K, epi, out, st), "gemm");
+  return MARCHE_OK;
+}
+
+int do_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void* cache_layer, const uint8_t* is_new,
+                 float* partial, void* o, cudaStream_t st) {
+  const marche_config& c = ctx->cfg;
+  MARCHE_TRY(launch_attention_simt(ctx->bf16, q, ld_q, c.batch, n, c.seq_len, c.n_heads, c.head_dim, cache_layer,
+                                   is_new, partial, o, st),
+             "attention");
+  return MARCHE_OK;
+}
+
+// The whole stack for M = B*nA rows.  active_idx == nullptr means every token (nA == S).
+int run_stack(marche_ctx* ctx, const float* hidden, void* kv_cache, const int32_t* active_idx, int nA,
+              const int32_t* new_idx, int n_new, const int32_t* excl_idx, int n_excl, float ratio,
+              float* hidden_out, int32_t* refresh_idx, int* n_refresh, void* workspace, size_t ws_bytes,
+              cudaStream_t st) {
+  const marche_config& c = ctx->cfg;
+  const int B = c.batch, S = c.seq_len, D = c.width, F = c.mlp_dim, H = c.n_heads, L = c.n_blocks;
+  if (!hidden || !kv_cache || !hidden_out || !workspace || hidden == hidden_out) return MARCHE_EINVAL;
+  if (nA < 1 || nA > S || n_new < 0 || n_new > nA || n_excl < 0 || n_new + n_excl > S) return MARCHE_EINVAL;
+  if ((n_new > 0 && !new_idx) || (n_excl > 0 && !excl_idx)) return MARCHE_EINVAL;
+  if (((uintptr_t)workspace & 255) != 0) return MARCHE_EINVAL;
+  const WsLayout w = ws_layout(ctx, nA);
+  if (ws_bytes < w.total) return MARCHE_EWORKSPACE;
+  const int k = refresh_idx ? refresh_count(ratio, S, S - n_new - n_excl) : 0;
+  if (n_refresh) *n_refresh = k;
+
+  char* ws = (char*)workspace;
+  float* scores = (float*)(ws + w.scores);
+  float* partial = (float*)(ws + w.partial);
+  uint8_t* cand = (uint8_t*)(ws + w.cand);
+  uint8_t* is_new = (uint8_t*)(ws + w.is_new);
+  float* x = (float*)(ws + w.x);
+  char* u = ws + w.u;
+  char* qkv = ws + w.qkv;
+  char* o = ws + w.o;
+  char* g = ws + w.g;
+  const int M = B * nA;
+  const size_t eb = ctx->eb;
+  const size_t layer_bytes = (size_t)2 * B * S * D * eb;
+
+  MARCHE_TRY(launch_step_flags(active_idx, nA, new_idx, n_new, excl_idx, n_excl, B, S, is_new, cand, st), "flags");
+  for (int l = 0; l < L; ++l) {
+    const marche_block_weights& bw = ctx->blocks[l];
+    char* cache_l = (char*)kv_cache + (size_t)l * layer_bytes;
+    if (l == 0)
+      MARCHE_TRY(launch_gather_layernorm(ctx->bf16, hidden, S, active_idx, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
+                                         x, u, st), "gather_layernorm");
+    else
+      MARCHE_TRY(launch_gather_layernorm(ctx->bf16, x, nA, nullptr, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
+                                         nullptr, u, st), "layernorm1");
+    int rc = do_linear(ctx, u, D, M, bw.w_qkv, bw.b_qkv, 3 * D, D, MARCHE_EPI_BIAS, qkv, st);
+    if (rc) return rc;
+    MARCHE_TRY(launch_scatter_kv(ctx->bf16, qkv + (size_t)D * eb, qkv + (size_t)2 * D * eb, 3 * D, active_idx, B, nA,
+                                 S, D, cache_l, st), "scatter_kv");
+    rc = do_attention(ctx, qkv, 3 * D, nA, cache_l, l == ctx->score_layer ? is_new : nullptr, partial, o, st);
+    if (rc) return rc;
+    rc = do_linear(ctx, o, D, M, bw.w_o, bw.b_o, D, D, MARCHE_EPI_BIAS_RESIDUAL, x, st);
+    if (rc) return rc;
+    MARCHE_TRY(launch_gather_layernorm(ctx->bf16, x, nA, nullptr, B, nA, D, bw.ln2_g, bw.ln2_b, ctx->eps, nullptr,
+                                       u, st), "layernorm2");
+    rc = do_linear(ctx, u, D, M, bw.w_fc1, bw.b_fc1, F, D, MARCHE_EPI_BIAS_GELU, g, st);
+    if (rc) return rc;
+    rc = do_linear(ctx, g, F, M, bw.w_fc2, bw.b_fc2, D, F, MARCHE_EPI_BIAS_RESIDUAL, x, st);
+    if (rc) return rc;
+  }
+  MARCHE_TRY(launch_scatter_rows(x, active_idx, B, nA, S, D, hidden_out, st), "scatter_rows");
+  MARCHE_TRY(launch_topk(partial, H, scores, cand, B, S, k, refresh_idx, st), "topk");
+  return MARCHE_OK;
+}
+
+std::pair<const void*, bool>* find_cache(marche_ctx* ctx, const void* p) {
+  for (auto& e : ctx->caches)
+    if (e.first == p) return &e;
+  return nullptr;
+}
+
+}  // namespace
+
+extern "C" {
+
+int marche_create(const marche_config* cfg, const marche_block_weights* blocks, marche_ctx** out) {
+  if (!cfg || !blocks || !out) return MARCHE_EINVAL;
+  *out = nullptr;
+  const marche_config& c = *cfg;
+  if (c.n_blocks < 1 || c.batch < 1 || c.seq_len < 1 || c.n_heads < 1 || c.head_dim < 1) return MARCHE_EINVAL;
+  if (c.dtype != MARCHE_F32 && c.dtype != MARCHE_BF16) return MARCHE_EINVAL;
+  if (c.width != c.n_heads * c.head_dim) return MARCHE_EINVAL;
+  if (c.width % 128 || c.width > 2048 || c.mlp_dim % 128 || c.mlp_dim < 128 || c.seq_len > 2048)
+    return MARCHE_ESHAPE;
+  if (c.head_dim % 16 || c.head_dim > 128) return MARCHE_ESHAPE;
+  if (c.dtype == MARCHE_BF16 && c.head_dim != 64 && c.head_dim != 80) return MARCHE_ESHAPE;
+  if (c.score_layer >= c.n_blocks) return MARCHE_EINVAL;
+  marche_ctx* ctx = new (std::nothrow) marche_ctx();
+  if (!ctx) return MARCHE_EINVAL;
+  ctx->cfg = c;
+  ctx->blocks.assign(blocks, blocks + c.n_blocks);
+  ctx->bf16 = c.dtype == MARCHE_BF16;
+  ctx->eb = ctx->bf16 ? 2 : 4;
+  ctx->eps = c.ln_eps > 0.f ? c.ln_eps : 1e-6f;
+  int sl = c.score_layer >= 0 ? c.score_layer : c.n_enc_blocks + 1;
+  if (sl >= c.n_blocks) sl = c.n_blocks - 1;
+  ctx->score_layer = sl;
+  const char* fs = getenv("MARCHE_FORCE_SIMT");
+  ctx->force_simt = fs && fs[0] == '1';
+  cudaError_t e = cudaGetDevice(&ctx->device);
+  if (e == cudaSuccess) e = cudaHostAlloc((void**)&ctx->status_host, 64, cudaHostAllocMapped);
+  if (e == cudaSuccess) {
+    memset(ctx->status_host, 0, 64);
+    e = cudaHostGetDevicePointer((void**)&ctx->status_dev, ctx->status_host, 0);
+  }
+  if (e != cudaSuccess) {
+    if (ctx->status_host) cudaFreeHost(ctx->status_host);
+    delete ctx;
+    return MARCHE_ECUDA;
+  }
+  *out = ctx;
+  return MARCHE_OK;
+}
+
+void marche_destroy(marche_ctx* ctx) {
+  if (!ctx) return;
+  if (ctx->status_host) cudaFreeHost(ctx->status_host);
+  delete ctx;
+}
+
+size_t marche_cache_bytes(const marche_ctx* ctx) {
+  if (!ctx) return 0;
+  const marche_config& c = ctx->cfg;
+  return (size_t)c.n_blocks * 2 * c.batch * c.seq_len * c.width * ctx->eb;
+}
+
+size_t marche_workspace_bytes(const marche_ctx* ctx, int max_active) {
+  if (!ctx || max_active < 1 || max_active > ctx->cfg.seq_len) return 0;
+  return ws_layout(ctx, max_active).total;
+}
+
+int marche_init_cache(marche_ctx* ctx, void* kv_cache, size_t bytes, marche_stream stream) {
+  if (!ctx || !kv_cache) return MARCHE_EINVAL;
+  if (bytes < marche_cache_bytes(ctx)) return MARCHE_EWORKSPACE;
+  MARCHE_TRY(cudaMemsetAsync(kv_cache, 0, marche_cache_bytes(ctx), (cudaStream_t)stream), "memset");
+  if (auto* e = find_cache(ctx, kv_cache)) e->second = false;
+  else ctx->caches.emplace_back(kv_cache, false);
+  return MARCHE_OK;
+}
+
+int marche_step(marche_ctx* ctx, const float* hidden, void* kv_cache, const int32_t* active_idx, int n_active,
+                const int32_t* new_idx, int n_new, const int32_t* exclude_idx, int n_excl, float refresh_ratio,
+                float* hidden_out, int32_t* refresh_idx, int* n_refresh, void* workspace, size_t workspace_bytes,
+                marche_stream stream) {
+  if (!ctx || !active_idx) return MARCHE_EINVAL;
+  auto* e = find_cache(ctx, kv_cache);
+  if (!e || !e->second) return MARCHE_ECACHE;
+  return run_stack(ctx, hidden, kv_cache, active_idx, n_active, new_idx, n_new, exclude_idx, n_excl, refresh_ratio,
+                   hidden_out, refresh_idx, n_refresh, workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+int marche_full_step(marche_ctx* ctx, const float* hidden, void* kv_cache, const int32_t* new_idx, int n_new,
+                     const int32_t* exclude_idx, int n_excl, float refresh_ratio, float* hidden_out,
+                     int32_t* refresh_idx, int* n_refresh, void* workspace, size_t workspace_bytes,
+                     marche_stream stream) {
+  if (!ctx) return MARCHE_EINVAL;
+  const int rc = run_stack(ctx, hidden, kv_cache, nullptr, ctx->cfg.seq_len, new_idx, n_new, exclude_idx, n_excl,
+                           refresh_ratio, hidden_out, refresh_idx, n_refresh, workspace, workspace_bytes,
+                           (cudaStream_t)stream);
+  if (rc == MARCHE_OK) {
+    if (auto* e = find_cache(ctx, kv_cache)) e->second = true;
+    else ctx->caches.emplace_back(kv_cache, true);
+  }
+  return rc;
+}
+
+int marche_select_refresh(marche_ctx* ctx, const float* scores, const int32_t* new_idx, int n_new,
+                          const int32_t* exclude_idx, int n_excl, int k, int32_t* refresh_idx, void* mask_scratch,
+                          marche_stream stream) {
+  if (!ctx || !scores || !mask_scratch || n_new < 0 || n_excl < 0 || k < 0) return MARCHE_EINVAL;
+  if ((n_new > 0 && !new_idx) || (n_excl > 0 && !exclude_idx)) return MARCHE_EINVAL;
+  const int B = ctx->cfg.batch, S = ctx->cfg.seq_len;
+  if (k > S - n_new - n_excl) return MARCHE_EINVAL;
+  if (k == 0) return MARCHE_OK;
+  if (!refresh_idx) return MARCHE_EINVAL;
+  cudaStream_t st = (cudaStream_t)stream;
+  MARCHE_TRY(launch_step_flags(nullptr, 0, new_idx, n_new, exclude_idx, n_excl, B, S, nullptr, (uint8_t*)mask_scratch,
+                               st), "flags");
+  MARCHE_TRY(launch_topk(nullptr, 0, const_cast<float*>(scores), (const uint8_t*)mask_scratch, B, S, k, refresh_idx,
+                         st), "topk");
+  return MARCHE_OK;
+}
+
+int marche_get_scores(marche_ctx* ctx, const void* workspace, float* scores_out, marche_stream stream) {
+  if (!ctx || !workspace || !scores_out) return MARCHE_EINVAL;
+  const size_t bytes = (size_t)ctx->cfg.batch * ctx->cfg.seq_len * sizeof(float);
+  MARCHE_TRY(cudaMemcpyAsync(scores_out, (const char*)workspace + ws_layout(ctx, 1).scores, bytes,
+                             cudaMemcpyDeviceToDevice, (cudaStream_t)stream), "memcpy");
+  return MARCHE_OK;
+}
+
+int marche_build_active(marche_ctx* ctx, const int32_t* new_idx, int n_new, const int32_t* prev_idx, int n_prev,
+                        const int32_t* refresh_idx, int n_refresh, int32_t* active_idx, marche_stream stream) {
+  if (!ctx || !active_idx || n_new < 0 || n_prev < 0 || n_refresh < 0) return MARCHE_EINVAL;
+  if ((n_new && !new_idx) || (n_prev && !prev_idx) || (n_refresh && !refresh_idx)) return MARCHE_EINVAL;
+  if (n_new + n_prev + n_refresh > ctx->cfg.seq_len) return MARCHE_EINVAL;
+  MARCHE_TRY(launch_build_active(new_idx, n_new, prev_idx, n_prev, refresh_idx, n_refresh, ctx->cfg.batch, active_idx,
+                                 (cudaStream_t)stream), "build_active");
+  return MARCHE_OK;
+}
+
+int marche_scatter_rows(marche_ctx* ctx, const float* rows, const int32_t* idx, int n, float* dst,
+                        marche_stream stream) {
+  if (!ctx || !rows || !dst || n < 0 || n > ctx->cfg.seq_len || (n && !idx)) return MARCHE_EINVAL;
+  MARCHE_TRY(launch_scatter_rows(rows, idx, ctx->cfg.batch, n, ctx->cfg.seq_len, ctx->cfg.width, dst,
+                                 (cudaStream_t)stream), "scatter_rows");
+  return MARCHE_OK;
+}
+
+int marche_validate_indices(marche_ctx* ctx, const int32_t* active_idx, int n_active, const int32_t* new_idx,
+                            int n_new, const int32_t* exclude_idx, int n_excl, marche_stream stream) {
+  if (!ctx || n_active < 0 || n_new < 0 || n_excl < 0) return MARCHE_EINVAL;
+  if ((n_active && !active_idx) || (n_new && !new_idx) || (n_excl && !exclude_idx)) return MARCHE_EINVAL;
+  const int S = ctx->cfg.seq_len;
+  if (n_active > S || n_new > S || n_excl > S) return MARCHE_EINDEX;
+  cudaStream_t st = (cudaStream_t)stream;
+  volatile int* flag = ctx->status_host + 8;   // second word group: index validation
+  *flag = 0;
+  MARCHE_TRY(launch_validate(n_active ? active_idx : nullptr, n_active, new_idx, n_new, exclude_idx, n_excl,
+                             ctx->cfg.batch, S, ctx->status_dev + 8, st), "validate");
+  MARCHE_TRY(cudaStreamSynchronize(st), "sync");
+  return *flag ? MARCHE_EINDEX : MARCHE_OK;
+}
+
+int marche_gather_layernorm(marche_ctx* ctx, const float* src, int src_rows, const int32_t* idx, int n,
+                            const float* gamma, const float* beta, float* x_out, void* u_out,
+                            marche_stream stream) {
+  if (!ctx || !src || !gamma || !beta || !u_out || n < 0 || src_rows < 1) return MARCHE_EINVAL;
+  if (!idx && n > src_rows) return MARCHE_EINVAL;
+  MARCHE_TRY(launch_gather_layernorm(ctx->bf16, src, src_rows, idx, ctx->cfg.batch, n, ctx->cfg.width, gamma, beta,
+                                     ctx->eps, x_out, u_out, (cudaStream_t)stream), "gather_layernorm");
+  return MARCHE_OK;
+}
+
+int marche_linear(marche_ctx* ctx, const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
+                  int epilogue, void* out, marche_stream stream) {
+  if (!ctx || !a || !w || !bias || !out || M < 0 || N < 1 || K < 1 || lda < K) return MARCHE_EINVAL;
+  if (epilogue < 0 || epilogue > 2) return MARCHE_EINVAL;
+  if (ctx->bf16 ? (N % 128 || K % 64 || lda % 8) : (N % 64 || K % 16 || lda % 4)) return MARCHE_ESHAPE;
+  return do_linear(ctx, a, lda, M, w, bias, N, K, epilogue, out, (cudaStream_t)stream);
+}
+
+int marche_scatter_kv(marche_ctx* ctx, const void* k, const void* v, int ld_kv, const int32_t* idx, int n,
+                      void* cache_layer, marche_stream stream) {
+  if (!ctx || !k || !v || !cache_layer || n < 0 || n > ctx->cfg.seq_len || ld_kv < ctx->cfg.width)
+    return MARCHE_EINVAL;
+  if (!idx && n != ctx->cfg.seq_len) return MARCHE_EINVAL;
+  MARCHE_TRY(launch_scatter_kv(ctx->bf16, k, v, ld_kv, idx, ctx->cfg.batch, n, ctx->cfg.seq_len, ctx->cfg.width,
+                               cache_layer, (cudaStream_t)stream), "scatter_kv");
+  return MARCHE_OK;
+}
+
+int marche_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void* cache_layer,
+                     const uint8_t* is_new, float* score_partial, void* o, marche_stream stream) {
+  if (!ctx || !q || !cache_layer || !o || n < 0 || n > ctx->cfg.seq_len || ld_q < ctx->cfg.width)
+    return MARCHE_EINVAL;
+  if (is_new && !score_partial) return MARCHE_EINVAL;
+  return do_attention(ctx, q, ld_q, n, cache_layer, is_new, score_partial, o, (cudaStream_t)stream);
+}
+
+const char* marche_strerror(int code) {
+  switch (code) {
+    case MARCHE_OK: return "ok";
+    case MARCHE_EINVAL: return "invalid argument";
+    case MARCHE_ESHAPE: return "unsupported shape";
+    case MARCHE_EWORKSPACE: return "workspace or cache buffer too small";
+    case MARCHE_ECACHE: return "cache-aware step on a cache that no full step has filled";
+    case MARCHE_EINDEX: return "invalid index set";
+    case MARCHE_ECUDA: return "CUDA error";
+    case MARCHE_ETIMEOUT: return "bounded device wait timed out";
+    default: return "unknown error";
+  }
+}
+
+const char* marche_last_error(const marche_ctx* ctx) { return ctx ? ctx->last_error.c_str() : ""; }
+
+int marche_device_status(const marche_ctx* ctx) { return ctx ? *(volatile int*)ctx->status_host : 0; }
+
+void marche_clear_device_status(marche_ctx* ctx) {
+  if (ctx) *(volatile int*)ctx->status_host = 0;
+}
+
+}  // extern "C"

@@ -1,0 +1,53 @@
+// Shared device helpers for the libmarche kernels (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+typedef __nv_bfloat16 bf16;
+
+#define MARCHE_DEVINL __device__ __forceinline__
+
+MARCHE_DEVINL float to_float(float v) { return v; }
+MARCHE_DEVINL float to_float(bf16 v) { return __bfloat162float(v); }
+
+template <typename T> MARCHE_DEVINL T from_float(float v);
+template <> MARCHE_DEVINL float from_float<float>(float v) { return v; }
+template <> MARCHE_DEVINL bf16 from_float<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+MARCHE_DEVINL uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+
+MARCHE_DEVINL float2 unpack_bf16x2(uint32_t u) {
+  __nv_bfloat162 p = *reinterpret_cast<__nv_bfloat162*>(&u);
+  return __bfloat1622float2(p);
+}
+
+MARCHE_DEVINL float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+MARCHE_DEVINL float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Exact (erf) GELU, the flavour the block uses.
+MARCHE_DEVINL float gelu_erf(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752440f)); }
+
+// Stores 4 consecutive outputs of type T starting at a 4-element aligned column.
+MARCHE_DEVINL void store4(float* p, float a, float b, float c, float d) {
+  *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
+}
+MARCHE_DEVINL void store4(bf16* p, float a, float b, float c, float d) {
+  uint2 u;
+  u.x = pack_bf16x2(a, b);
+  u.y = pack_bf16x2(c, d);
+  *reinterpret_cast<uint2*>(p) = u;
+}

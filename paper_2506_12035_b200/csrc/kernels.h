@@ -1,0 +1,51 @@
+// Host-side launch wrappers, one per kernel; raw device pointers and a stream.
+// Every wrapper only enqueues work and returns the launch's cudaError_t.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace marche {
+
+// K1: gather + LayerNorm.  rows = B*n; src row of (b, j) is src[b][idx ? idx[b][j] : j].
+cudaError_t launch_gather_layernorm(bool bf16_out, const float* src, int src_rows, const int32_t* idx,
+                                    int B, int n, int D, const float* gamma, const float* beta, float eps,
+                                    float* x_out, void* u_out, cudaStream_t st);
+
+// K5: K/V write-back into one block's cache slice [2][B][S][D]; idx NULL = identity.
+cudaError_t launch_scatter_kv(bool bf16_t, const void* k, const void* v, int ld_kv, const int32_t* idx,
+                              int B, int n, int S, int D, void* cache_layer, cudaStream_t st);
+
+// fp32 row scatter dst[b][idx ? idx[b][j] : j] = rows[b][j].
+cudaError_t launch_scatter_rows(const float* rows, const int32_t* idx, int B, int n, int S, int D,
+                                float* dst, cudaStream_t st);
+
+// a0 prologue: is_new[b][j] (may be NULL with n_active = 0) and the candidate mask cand[b][t].
+cudaError_t launch_step_flags(const int32_t* active_idx, int n_active, const int32_t* new_idx, int n_new,
+                              const int32_t* excl_idx, int n_excl, int B, int S, uint8_t* is_new,
+                              uint8_t* cand, cudaStream_t st);
+
+cudaError_t launch_build_active(const int32_t* a, int na, const int32_t* b, int nb, const int32_t* c, int nc,
+                                int B, int32_t* out, cudaStream_t st);
+
+// Index validation; *status (device or mapped host int) is set non-zero on a violation.
+cudaError_t launch_validate(const int32_t* active_idx, int n_active, const int32_t* new_idx, int n_new,
+                            const int32_t* excl_idx, int n_excl, int B, int S, int* status, cudaStream_t st);
+
+// K4: optional fixed-order head reduction of score partials [B][H][S] into scores [B][S],
+// then top-k among cand (k may be 0: reduction only).
+cudaError_t launch_topk(const float* partial, int H, float* scores, const uint8_t* cand, int B, int S, int k,
+                        int32_t* refresh_idx, cudaStream_t st);
+
+// K2 (fp32 SIMT and bf16 SIMT bring-up path).
+cudaError_t launch_gemm_simt(bool bf16_t, const void* a, int lda, int M, const void* w, const float* bias,
+                             int N, int K, int epilogue, void* out, cudaStream_t st);
+
+// K3 (SIMT): attention of n queries per sample over all S cache rows.
+cudaError_t launch_attention_simt(bool bf16_t, const void* q, int ld_q, int B, int n, int S, int H, int dh,
+                                  const void* cache_layer, const uint8_t* is_new, float* score_partial,
+                                  void* o, cudaStream_t st);
+size_t attention_simt_smem(int S, int dh);
+
+}  // namespace marche

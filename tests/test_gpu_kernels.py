@@ -1,0 +1,265 @@
+"""Per-kernel parity: each C-ABI kernel call against the matching oracle sub-step on the
+same seeded inputs (small and odd shapes spanning several tiles and ragged tails)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import marche_oracle as orc
+from helpers import (TOL, assert_close, dev, host, idx_dev, make_model, max_abs, rel_l2)
+
+pytestmark = pytest.mark.gpu
+
+
+def model_for(dtype, D, H, F, S, B, L=1):
+    cfg = synth.CONFIGS["tiny"].replace(L=L, E=0, D=D, H=H, F=F, S=S, B=B, dtype=dtype, n_buffer=0)
+    blocks = synth.make_weights(cfg)
+    return cfg, blocks, make_model(cfg, blocks)
+
+
+def tdt(dtype):
+    return torch.bfloat16 if dtype == "bf16" else torch.float32
+
+
+def quant(a, dtype):
+    """What the device holds for an operand of the compute type."""
+    return synth.round_to_bf16(a).astype(np.float64) if dtype == "bf16" else np.asarray(a, np.float32).astype(np.float64)
+
+
+# ------------------------------------------------------------------ K1 gather + LayerNorm
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("D,H", [(256, 4), (768, 12), (1024, 16), (1280, 16)])
+@pytest.mark.parametrize("n", [1, 2, 41, 68])
+def test_gather_layernorm(dtype, D, H, n):
+    S, B = 68, 3
+    cfg, blocks, m = model_for(dtype, D, H, 128, S, B)
+    rng = np.random.default_rng(n + D)
+    hidden = rng.standard_normal((B, S, D)).astype(np.float32)
+    hidden[0] += 100.0                                   # large mean: variance cancellation
+    patterns = [np.stack([rng.permutation(S)[:n] for _ in range(B)]),
+                np.tile(np.arange(S - 1, S - 1 - n, -1), (B, 1))]
+    g, be = blocks[0]["ln1_g"], blocks[0]["ln1_b"]
+    for idx in patterns:
+        x_out = torch.full((B * n, D), -7.0, device="cuda")
+        u_out = torch.zeros(B * n, D, dtype=tdt(dtype), device="cuda")
+        m.gather_layernorm(dev(hidden), idx_dev(idx), n, dev(g), dev(be), x_out, u_out)
+        X = np.stack([hidden[b, idx[b]] for b in range(B)]).reshape(B * n, D)
+        assert np.array_equal(x_out.cpu().numpy(), X)                       # the gather is a copy: exact
+        want = orc.layer_norm(X.astype(np.float64), g.astype(np.float64), be.astype(np.float64), cfg.ln_eps)
+        assert_close(host(u_out), want, dtype, "LN", scale=1.0 if dtype == "bf16" else 10.0)
+    # identity index (idx NULL), no compact copy
+    u_out = torch.zeros(B * n, D, dtype=tdt(dtype), device="cuda")
+    m.gather_layernorm(dev(hidden), None, n, dev(g), dev(be), None, u_out)
+    want = orc.layer_norm(hidden[:, :n].reshape(B * n, D).astype(np.float64), g.astype(np.float64),
+                          be.astype(np.float64), cfg.ln_eps)
+    assert_close(host(u_out), want, dtype, "LN identity", scale=1.0 if dtype == "bf16" else 10.0)
+
+
+# ------------------------------------------------------------------ K2 projections
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("M", [1, 24, 62, 129, 300])
+@pytest.mark.parametrize("N,K", [(768, 256), (256, 256), (1024, 256), (256, 1024), (384, 128), (128, 320)])
+def test_linear_all_epilogues(dtype, M, N, K):
+    cfg, blocks, m = model_for(dtype, 256, 4, 1024, 68, 2)
+    rng = np.random.default_rng(M * 7 + N + K)
+    a = rng.standard_normal((M, K)).astype(np.float32)
+    w = (rng.standard_normal((N, K)) * 0.05).astype(np.float32)
+    bias = rng.standard_normal(N).astype(np.float32)
+    aq, wq = quant(a, dtype), quant(w, dtype)
+    acc = orc.linear(aq, wq, bias.astype(np.float64))
+    a_d, w_d, b_d = dev(a, tdt(dtype)), dev(w, tdt(dtype)), dev(bias)
+    ma, rl = TOL[dtype]
+    # bias
+    out = torch.zeros(M, N, dtype=tdt(dtype), device="cuda")
+    m.linear(a_d, w_d, b_d, 0, out)
+    assert rel_l2(host(out), acc) <= (4e-3 if dtype == "bf16" else 1e-6)
+    assert max_abs(host(out), acc) <= (3e-2 if dtype == "bf16" else 1e-4)
+    # bias + residual (fp32 read-modify-write)
+    res = rng.standard_normal((M, N)).astype(np.float32)
+    out = dev(res)
+    m.linear(a_d, w_d, b_d, 1, out)
+    assert max_abs(host(out), acc + res) <= 1e-4 * max(1.0, math.sqrt(K / 256))
+    # bias + GELU
+    out = torch.zeros(M, N, dtype=tdt(dtype), device="cuda")
+    m.linear(a_d, w_d, b_d, 2, out)
+    want = orc.gelu(acc)
+    assert rel_l2(host(out), want) <= (4e-3 if dtype == "bf16" else 1e-6)
+    assert max_abs(host(out), want) <= (3e-2 if dtype == "bf16" else 1e-4)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_linear_strided_input_and_row_guard(dtype):
+    """a is a column slice of a wider matrix (lda > K); rows >= M of `out` stay untouched."""
+    cfg, blocks, m = model_for(dtype, 256, 4, 1024, 68, 2)
+    rng = np.random.default_rng(5)
+    M, N, K = 70, 256, 256
+    wide = rng.standard_normal((M, 3 * K)).astype(np.float32)
+    w = (rng.standard_normal((N, K)) * 0.05).astype(np.float32)
+    bias = rng.standard_normal(N).astype(np.float32)
+    wide_d = dev(wide, tdt(dtype))
+    out = torch.full((M + 60, N), 5.0, dtype=tdt(dtype), device="cuda")
+    m.linear(wide_d[:, K:2 * K], dev(w, tdt(dtype)), dev(bias), 0, out, M=M, lda=3 * K)
+    want = orc.linear(quant(wide[:, K:2 * K], dtype), quant(w, dtype), bias.astype(np.float64))
+    assert rel_l2(host(out[:M]), want) <= (4e-3 if dtype == "bf16" else 1e-6)
+    assert (host(out[M:]) == 5.0).all()
+
+
+# ------------------------------------------------------------------ K5 scatter
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("n", [1, 7, 41])
+def test_scatter_kv_and_untouched_rows(dtype, n):
+    S, B, D = 68, 3, 256
+    cfg, blocks, m = model_for(dtype, D, 4, 128, S, B)
+    rng = np.random.default_rng(n)
+    qkv = dev(rng.standard_normal((B * n, 3 * D)).astype(np.float32), tdt(dtype))
+    cache = dev(rng.standard_normal((2, B, S, D)).astype(np.float32), tdt(dtype))
+    before = cache.clone()
+    idx = np.stack([rng.permutation(S)[:n] for _ in range(B)]).astype(np.int32)
+    m.scatter_kv(qkv[:, D:], qkv[:, 2 * D:], 3 * D, idx_dev(idx), n, cache)
+    torch.cuda.synchronize()
+    want = before.clone()
+    q3 = qkv.view(B, n, 3 * D)
+    for b in range(B):
+        want[0, b, torch.as_tensor(idx[b], dtype=torch.long)] = q3[b, :, D:2 * D]
+        want[1, b, torch.as_tensor(idx[b], dtype=torch.long)] = q3[b, :, 2 * D:]
+    assert torch.equal(cache, want)                                     # byte-identical everywhere
+
+
+def test_scatter_rows_and_build_active():
+    S, B, D = 68, 3, 256
+    cfg, blocks, m = model_for("f32", D, 4, 128, S, B)
+    rng = np.random.default_rng(0)
+    rows = dev(rng.standard_normal((B, 5, D)).astype(np.float32))
+    idx = np.stack([rng.permutation(S)[:5] for _ in range(B)]).astype(np.int32)
+    dst = torch.full((B, S, D), 3.0, device="cuda")
+    m.scatter_rows(rows, idx_dev(idx), dst)
+    want = torch.full((B, S, D), 3.0, device="cuda")
+    for b in range(B):
+        want[b, torch.as_tensor(idx[b], dtype=torch.long)] = rows[b]
+    assert torch.equal(dst, want)
+    G, N, R = idx[:, :2], idx[:, 2:3], idx[:, 3:]
+    act = torch.zeros(B, 5, dtype=torch.int32, device="cuda")
+    m.build_active(idx_dev(G), idx_dev(N), idx_dev(R), 2, act)
+    assert np.array_equal(act.cpu().numpy(), orc.active_set(G, N, R))
+    act2 = torch.zeros(B, 2, dtype=torch.int32, device="cuda")
+    m.build_active(idx_dev(G), None, None, 0, act2)
+    assert np.array_equal(act2.cpu().numpy(), G)
+
+
+# ------------------------------------------------------------------ K3 attention (+ scores)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("S", [68, 320])
+@pytest.mark.parametrize("dh,H", [(64, 4), (80, 2)])
+@pytest.mark.parametrize("n,nG", [(1, 1), (2, 0), (12, 7), (41, 25), (77, 77)])
+def test_attention_and_score_partials(dtype, S, dh, H, n, nG):
+    if n > S:
+        pytest.skip("n > S")
+    B, D = 2, dh * H
+    if D % 128:
+        H = {64: 4, 80: 8}[dh]
+        D = dh * H
+    cfg, blocks, m = model_for(dtype, D, H, 128, S, B)
+    rng = np.random.default_rng(S + n + dh)
+    gain = 3.0                                                       # logits of order a few units
+    q = (rng.standard_normal((B * n, 3 * D)) * gain).astype(np.float32)
+    cache = rng.standard_normal((2, B, S, D)).astype(np.float32)
+    flags = np.zeros((B, n), dtype=np.uint8)
+    for b in range(B):
+        flags[b, rng.permutation(n)[:nG]] = 1
+    q_d = dev(q, tdt(dtype))
+    o = torch.zeros(B * n, D, dtype=tdt(dtype), device="cuda")
+    partial = torch.full((B, H, S), -1.0, device="cuda")
+    m.attention(q_d, 3 * D, n, dev(cache, tdt(dtype)), dev(flags), partial, o)
+    qq, cc = quant(q, dtype), quant(cache, dtype)
+    want_o = np.zeros((B * n, D))
+    want_p = np.zeros((B, H, S))
+    for b in range(B):
+        for h in range(H):
+            c = slice(h * dh, (h + 1) * dh)
+            z, p = orc.softmax_attention(qq[b * n:(b + 1) * n, c], cc[0, b][:, c], cc[1, b][:, c])
+            want_o[b * n:(b + 1) * n, c] = z
+            want_p[b, h] = p[flags[b].astype(bool)].sum(axis=0)
+    got_o, got_p = host(o), host(partial)
+    assert rel_l2(got_o, want_o) <= (8e-3 if dtype == "bf16" else 1e-5)
+    assert max_abs(got_o, want_o) <= (3e-2 if dtype == "bf16" else 1e-4)
+    assert max_abs(got_p, want_p) <= (2e-2 if dtype == "bf16" else 1e-5) * max(1, nG) / 8 + 1e-6
+    assert np.allclose(got_p.sum(-1), nG, rtol=(5e-3 if dtype == "bf16" else 1e-5), atol=1e-6)   # each row sums to 1
+    # scores off: partial buffer untouched
+    partial2 = torch.full((B, H, S), -1.0, device="cuda")
+    m.attention(q_d, 3 * D, n, dev(cache, tdt(dtype)), None, partial2, o)
+    assert (partial2 == -1.0).all()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_attention_uniform_and_peaked(dtype):
+    S, B, H, dh, n = 68, 2, 4, 64, 5
+    D = H * dh
+    cfg, blocks, m = model_for(dtype, D, H, 128, S, B)
+    rng = np.random.default_rng(1)
+    cache = rng.standard_normal((2, B, S, D)).astype(np.float32)
+    flags = np.ones((B, n), dtype=np.uint8)
+    # q = 0 -> uniform weights: o = mean of V, partial = n / S
+    o = torch.zeros(B * n, D, dtype=tdt(dtype), device="cuda")
+    partial = torch.zeros(B, H, S, device="cuda")
+    m.attention(torch.zeros(B * n, D, dtype=tdt(dtype), device="cuda"), D, n, dev(cache, tdt(dtype)), dev(flags),
+                partial, o)
+    vm = quant(cache, dtype)[1].mean(axis=1)
+    assert max_abs(host(o).reshape(B, n, D), np.repeat(vm[:, None], n, 1)) <= (4e-3 if dtype == "bf16" else 1e-5)
+    assert np.allclose(host(partial), n / S, rtol=1e-3 if dtype == "bf16" else 1e-5)
+    # q = 64 * k_t -> one-hot on key t: o = V[t]; no inf/nan
+    tsel = rng.integers(0, S, size=(B, n))
+    kq = quant(cache, dtype)
+    q = np.stack([kq[0, b, tsel[b]] for b in range(B)]).reshape(B * n, D) * 64.0
+    m.attention(dev(q.astype(np.float32), tdt(dtype)), D, n, dev(cache, tdt(dtype)), dev(flags), partial, o)
+    got = host(o).reshape(B, n, D)
+    assert np.isfinite(got).all()
+    for b in range(B):
+        assert max_abs(got[b], kq[1, b, tsel[b]]) <= (2e-2 if dtype == "bf16" else 1e-4)
+    assert np.allclose(host(partial).sum(-1), n, rtol=1e-3)
+
+
+# ------------------------------------------------------------------ K4 top-k (bit-exact)
+@pytest.mark.parametrize("S,k", [(5, 2), (68, 7), (320, 32), (320, 0), (320, 311), (1088, 109), (1088, 1)])
+def test_select_refresh_bit_exact(S, k):
+    B = 4
+    cfg, blocks, m = model_for("f32", 128, 2, 128, S, B)
+    rng = np.random.default_rng(S * 3 + k)
+    n_new, n_excl = (2, 3) if S > 5 else (1, 1)
+    kinds = [rng.random((B, S)), np.ones((B, S)), rng.integers(0, 3, (B, S)).astype(float),
+             rng.random((B, S)) * 1e-42, np.exp(rng.uniform(-80, 10, (B, S))), np.zeros((B, S))]
+    kinds[5][:, ::2] = -0.0
+    mask = torch.empty(B * S, dtype=torch.uint8, device="cuda")
+    for sc in kinds:
+        sc = sc.astype(np.float32)
+        perm = np.stack([rng.permutation(S) for _ in range(B)]).astype(np.int32)
+        for new, excl in ((perm[:, :n_new], perm[:, n_new:n_new + n_excl]), (perm[:, :n_new], None),
+                          (np.tile(np.arange(n_new, dtype=np.int32), (B, 1)), np.tile(np.arange(S - n_excl, S, dtype=np.int32), (B, 1)))):
+            kk = min(k, S - n_new - (0 if excl is None else n_excl))
+            out = torch.full((B, max(kk, 1)), -1, dtype=torch.int32, device="cuda")
+            m.select_refresh(dev(sc), idx_dev(new), None if excl is None else idx_dev(excl), kk, out, mask)
+            want = orc.select_refresh(sc, new, excl, kk)
+            if kk:
+                assert np.array_equal(out.cpu().numpy(), want)
+            else:
+                assert (out.cpu().numpy() == -1).all()
+
+
+def test_validate_indices():
+    from paper_2506_12035_b200.binding import MarcheError
+    S, B = 68, 2
+    cfg, blocks, m = model_for("f32", 128, 2, 128, S, B)
+    act = np.array([[1, 2, 3, 4], [5, 6, 7, 8]], np.int32)
+    new = act[:, :2]
+    excl = np.array([[9], [10]], np.int32)
+    m.validate_indices(idx_dev(act), idx_dev(new), idx_dev(excl))
+    for bad_act, bad_new, bad_excl in [
+        (np.array([[1, 2, 3, 3], [5, 6, 7, 8]], np.int32), new, excl),            # duplicate
+        (np.array([[1, 2, 3, 68], [5, 6, 7, 8]], np.int32), new, excl),           # out of range
+        (act, np.array([[1, 9], [5, 6]], np.int32), None),                         # new not in active
+        (act, new, np.array([[2], [10]], np.int32)),                               # exclude overlaps new
+    ]:
+        with pytest.raises(MarcheError) as e:
+            m.validate_indices(idx_dev(bad_act), idx_dev(bad_new), None if bad_excl is None else idx_dev(bad_excl))
+        assert e.value.code == -5

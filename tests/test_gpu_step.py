@@ -1,0 +1,196 @@
+"""End-to-end parity of marche_step / marche_full_step with the CPU oracle, teacher-forced:
+both sides are driven with the oracle's index sets at every step, and per step the
+active rows of hidden_out, the relevance scores and (at the end) every cache layer are
+compared.  Plus the invariants that hold at any size and the error behaviour."""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import marche_oracle as orc
+from paper_2506_12035_b200.binding import MarcheError
+from paper_2506_12035_b200.generation import Generation
+from helpers import TOL, assert_close, cache_to_oracle_layout, dev, host, idx_dev, make_model, max_abs, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+CASES = {
+    # the fp32 configuration of the benchmark list, whole 8-step generation
+    "tiny_f32": synth.CONFIGS["tiny"],
+    # same stack in bf16
+    "tiny_bf16": synth.CONFIGS["tiny"].replace(dtype="bf16"),
+    # MAR-B-shaped rows (D 768, 12 heads, S 320), cut down in depth, batch and steps
+    "marb_slice": synth.CONFIGS["mar_b"].replace(L=3, E=1, B=4, T=6),
+    # head_dim 80 (MAR-H-shaped rows)
+    "marh_slice": synth.CONFIGS["mar_h"].replace(L=2, E=0, B=2, T=4),
+}
+
+
+def oracle_run(cfg, blocks, hidden0, ratio, mode="marche"):
+    sets = synth.new_token_sets(cfg, synth.generation_orders(cfg))
+    rep = lambda t, n: synth.replacement_rows(cfg, t, n)
+    log, cache = orc.generate(blocks, hidden0, sets, rep, ratio, n_heads=cfg.H, score_layer=cfg.score_layer,
+                              ln_eps=cfg.ln_eps, mode=mode)
+    return sets, log, cache
+
+
+def gpu_generation(cfg, blocks, sets, ratio):
+    m = make_model(cfg, blocks)
+    rows = [dev(synth.replacement_rows(cfg, t, sets[t].shape[1])) for t in range(cfg.T)]
+    return m, Generation(m, sets, ratio, rows)
+
+
+@pytest.mark.parametrize("case", list(CASES))
+@pytest.mark.parametrize("ratio", [0.10, 0.0])
+def test_teacher_forced_generation(case, ratio):
+    cfg = CASES[case]
+    if ratio == 0.0 and case != "tiny_bf16":
+        pytest.skip("zero-refresh variant runs on one case")
+    blocks = synth.make_weights(cfg)
+    hidden0 = synth.make_hidden(cfg)
+    sets, log, cache = oracle_run(cfg, blocks, hidden0, ratio)
+    m, gen = gpu_generation(cfg, blocks, sets, ratio)
+    forced = [idx_dev(rec["refresh"]) for rec in log]
+    glog = gen.run(dev(hidden0), record=True, forced_refresh=forced)
+    assert m.device_status() == 0
+    mask = torch.empty(cfg.B * cfg.S, dtype=torch.uint8, device="cuda")
+    for rec, g in zip(log, glog):
+        A = rec["active"]
+        assert g["n_active"] == A.shape[1]
+        if g["active"] is not None:
+            assert np.array_equal(g["active"], A)                      # device-built A = G u N u R
+        for b in range(cfg.B):
+            assert_close(g["hidden_out"][b, A[b]], rec["hidden_out"][b, A[b]], cfg.dtype,
+                         "%s step %d hidden_out" % (case, rec["t"]))
+        nG = rec["new"].shape[1]
+        unit = cfg.H * nG / cfg.S                                      # mean score
+        assert max_abs(g["scores"], rec["scores"]) <= (5e-2 if cfg.dtype == "bf16" else 1e-4) * unit
+        assert np.allclose(g["scores"].sum(-1), cfg.H * nG, rtol=1e-3)
+        # selection: fed the oracle's fp32 scores, the device's top-k is bit-exact
+        k = rec["refresh"].shape[1]
+        if k:
+            out = torch.empty(cfg.B, k, dtype=torch.int32, device="cuda")
+            excl = rec["exclude"]
+            m.select_refresh(dev(rec["scores"]), idx_dev(rec["new"]), idx_dev(excl) if excl.shape[1] else None,
+                             k, out, mask)
+            assert np.array_equal(out.cpu().numpy(), rec["refresh"])
+    K, V = cache_to_oracle_layout(gen.cache)
+    assert_close(K, cache.K, cfg.dtype, case + " cache K")
+    assert_close(V, cache.V, cfg.dtype, case + " cache V")
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_invariants_untouched_rows_full_equivalence_reproducibility(dtype):
+    cfg = synth.CONFIGS["tiny"].replace(dtype=dtype, B=3)
+    blocks = synth.make_weights(cfg)
+    m = make_model(cfg, blocks)
+    rng = np.random.default_rng(0)
+    B, S, D = cfg.B, cfg.S, cfg.D
+    hidden = dev(synth.make_hidden(cfg))
+    cache = m.alloc_cache()
+    ws = m.alloc_workspace(S)
+    out_full = torch.zeros(B, S, D, device="cuda")
+    refresh = torch.zeros(B, S, dtype=torch.int32, device="cuda")
+    A = np.stack([rng.permutation(S)[:9] for _ in range(B)]).astype(np.int32)
+    G = A[:, :3]
+    # a step on a never-filled cache is an error and enqueues nothing
+    m.init_cache(cache)
+    with pytest.raises(MarcheError) as e:
+        m.step(hidden, cache, idx_dev(A), idx_dev(G), None, 0.1, out_full, refresh, ws)
+    assert e.value.code == -4
+    k_full = m.full_step(hidden, cache, idx_dev(G), None, 0.1, out_full, refresh, ws)
+    sc_full = torch.empty(B, S, device="cuda")
+    m.get_scores(ws, sc_full)
+    cache_full = cache.clone()
+
+    # P5: rows outside A are byte-identical after a cache-aware step (sentinel in hidden_out)
+    hidden2 = hidden.clone()
+    for b in range(B):
+        hidden2[b, torch.as_tensor(A[b], dtype=torch.long)] += 0.5
+    out = torch.full((B, S, D), 777.0, device="cuda")
+    m.step(hidden2, cache, idx_dev(A), idx_dev(G), None, 0.1, out, refresh, ws)
+    torch.cuda.synchronize()
+    for b in range(B):
+        rest = torch.as_tensor(np.setdiff1d(np.arange(S), A[b]), dtype=torch.long)
+        act = torch.as_tensor(A[b], dtype=torch.long)
+        assert torch.equal(cache[:, :, b, rest], cache_full[:, :, b, rest])
+        assert not torch.equal(cache[:, :, b, act], cache_full[:, :, b, act])
+        assert (out[b, rest] == 777.0).all() and (out[b, act] != 777.0).all()
+
+    # P1/P3: active = every token (any order) reproduces the full step
+    cache2 = m.alloc_cache()
+    m.init_cache(cache2)
+    out_b = torch.zeros(B, S, D, device="cuda")
+    m.full_step(hidden, cache2, idx_dev(G), None, 0.1, out_b, refresh, ws)
+    perm = np.stack([rng.permutation(S) for _ in range(B)]).astype(np.int32)
+    out_c = torch.zeros(B, S, D, device="cuda")
+    refresh_c = torch.zeros(B, S, dtype=torch.int32, device="cuda")
+    k_c = m.step(hidden, cache2, idx_dev(perm), idx_dev(G), None, 0.1, out_c, refresh_c, ws)
+    sc_c = torch.empty(B, S, device="cuda")
+    m.get_scores(ws, sc_c)
+    tol = 2e-2 if dtype == "bf16" else 1e-5
+    assert max_abs(host(out_c), host(out_full)) <= tol
+    assert max_abs(host(cache2), host(cache_full)) <= tol
+    assert max_abs(host(sc_c), host(sc_full)) <= 1e-3 and k_c == k_full
+
+    # run-to-run bit reproducibility (scores use a fixed-order reduction, no atomics)
+    res = []
+    for _ in range(2):
+        c3 = cache_full.clone()
+        m.init_cache(c3)
+        o3 = torch.zeros(B, S, D, device="cuda")
+        r3 = torch.zeros(B, S, dtype=torch.int32, device="cuda")
+        m.full_step(hidden, c3, idx_dev(G), None, 0.1, o3, r3, ws)
+        m.step(hidden2, c3, idx_dev(A), idx_dev(G), None, 0.1, o3, r3, ws)
+        s3 = torch.empty(B, S, device="cuda")
+        m.get_scores(ws, s3)
+        res.append((o3.clone(), c3, s3, r3.clone()))
+    for x, y in zip(*res):
+        assert torch.equal(x, y)
+
+
+def test_full_ratio_equals_full_recompute():
+    """Refresh ratio 100 %: every step's active set is all tokens, so the cache-aware
+    generation equals the full-recompute generation (Appendix A)."""
+    cfg = synth.CONFIGS["tiny"].replace(dtype="bf16")
+    blocks = synth.make_weights(cfg)
+    hidden0 = dev(synth.make_hidden(cfg))
+    sets = synth.new_token_sets(cfg, synth.generation_orders(cfg))
+    m, gen = gpu_generation(cfg, blocks, sets, 1.0)
+    log_m = gen.run(hidden0, mode="marche", record=True)
+    cache_m = gen.cache.clone()
+    log_f = gen.run(hidden0, mode="full", record=True)
+    for a, f in zip(log_m, log_f):
+        assert a["n_active"] == cfg.S
+        assert max_abs(a["hidden_out"], f["hidden_out"]) <= 2e-2
+        assert rel_l2(a["hidden_out"], f["hidden_out"]) <= 2e-3
+    assert max_abs(host(cache_m), host(gen.cache)) <= 2e-2
+
+
+def test_argument_errors():
+    cfg = synth.CONFIGS["tiny"]
+    blocks = synth.make_weights(cfg)
+    m = make_model(cfg, blocks)
+    B, S, D = cfg.B, cfg.S, cfg.D
+    hidden = dev(synth.make_hidden(cfg))
+    out = torch.zeros(B, S, D, device="cuda")
+    cache = m.alloc_cache()
+    m.init_cache(cache)
+    small_ws = m.alloc_workspace(4)
+    refresh = torch.zeros(B, S, dtype=torch.int32, device="cuda")
+    G = idx_dev(np.array([[4, 5], [6, 7]]))
+    with pytest.raises(MarcheError) as e:
+        m.full_step(hidden, cache, G, None, 0.1, out, refresh, small_ws)
+    assert e.value.code == -3
+    ws = m.alloc_workspace(S)
+    with pytest.raises(MarcheError) as e:
+        m.full_step(hidden, cache, G, None, 0.1, hidden, refresh, ws)          # out aliases in
+    assert e.value.code == -1
+    m.full_step(hidden, cache, G, None, 0.1, out, refresh, ws)
+    with pytest.raises(MarcheError) as e:                                       # n_new > n_active
+        m.step(hidden, cache, idx_dev(np.array([[4], [6]])), G, None, 0.1, out, refresh, ws)
+    assert e.value.code == -1
+    from paper_2506_12035_b200.binding import Marche, upload_weights
+    with pytest.raises(MarcheError) as e:                                       # width not a multiple of 128
+        Marche(L=1, E=0, D=192, H=3, F=128, S=8, B=1, dtype="f32", weights=upload_weights(blocks[:1], "f32"))
+    assert e.value.code == -2
