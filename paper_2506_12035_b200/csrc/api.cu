@@ -83,7 +83,12 @@ int refresh_count(float ratio, int S, int n_cand) {
 
 int do_linear(marche_ctx* ctx, const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
               int epi, void* out, cudaStream_t st) {
-  MARCHE_TRY(launch_gemm_simt(ctx->bf16, a, lda, M, w, bias, N, K, epi, out, st), "gemm");
+  const bool tc = ctx->bf16 && !ctx->force_simt && N % 128 == 0 && K % 64 == 0 && lda % 8 == 0 &&
+                  (((uintptr_t)a | (uintptr_t)w | (uintptr_t)out) & 15) == 0;
+  if (tc)
+    MARCHE_TRY(launch_gemm_tcgen05(a, lda, M, w, bias, N, K, epi, out, ctx->status_dev, st), "gemm_tcgen05");
+  else
+    MARCHE_TRY(launch_gemm_simt(ctx->bf16, a, lda, M, w, bias, N, K, epi, out, st), "gemm");
   return MARCHE_OK;
 }
 

@@ -1,0 +1,299 @@
+// K2: out = epilogue(a * w^T + bias) on the 5th-generation tensor cores.
+//
+// The QKV, output and MLP projections of the active rows (Algorithm 1 lines 5 and 9)
+// are dense bf16 contractions, so they run as a persistent, warp-specialised tcgen05
+// kernel: one CTA per SM walks over 128 x BN output tiles;
+//   warp 0   (one lane)  TMA producer: 128x64 A tile and BNx64 W tile per K step into a
+//                        shared-memory ring (128-byte swizzle), completion on mbarriers
+//   warp 1   (one lane)  issues tcgen05.mma (M 128, N BN, K 16; bf16 in, fp32 accumulate
+//                        in TMEM), frees ring slots and publishes accumulators with
+//                        tcgen05.commit
+//   warps 2-5            epilogue: tcgen05.ld of the accumulator (thread = output row),
+//                        bias / GELU / fp32 residual, stores
+// The accumulator is double-buffered in TMEM (2 x BN columns) so the epilogue of tile i
+// overlaps the MMAs of tile i+1.  Rows beyond M are zero-filled by TMA on load and
+// masked on store, so M needs no padding.  Every mbarrier wait is bounded; on a
+// give-up the kernel records a status code and drains instead of hanging.
+#include <cuda.h>
+
+#include "kernels.h"
+#include "sm100_ptx.cuh"
+
+namespace marche {
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;                    // one 128-byte swizzle row of bf16
+constexpr int kGemmThreads = 192;
+constexpr int A_BYTES = BM * BK * 2;      // 16 KB
+
+template <int BN> struct GemmCfg {
+  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int STAGES = (BN == 256) ? 4 : 6;
+  static constexpr int RING_BYTES = STAGES * (A_BYTES + B_BYTES);
+  static constexpr int SMEM_BYTES = RING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int TMEM_COLS = 2 * BN;
+};
+
+enum { ST_PRODUCER = 0x11, ST_MMA = 0x12, ST_EPILOGUE = 0x13 };
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
+                    int M, int N, int K, const float* __restrict__ bias, void* __restrict__ out_,
+                    int* __restrict__ status) {
+  using Cfg = GemmCfg<BN>;
+  constexpr int STAGES = Cfg::STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = ptx::smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;             // swizzled tiles need 1024-byte alignment
+  const uint32_t a_base = base;
+  const uint32_t w_base = base + STAGES * A_BYTES;
+  const uint32_t bar_base = base + Cfg::RING_BYTES;         // 8-byte barriers
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+  uint8_t* gen_base = smem_raw + (base - raw);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + Cfg::RING_BYTES + 8 * (2 * STAGES + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + Cfg::RING_BYTES + 8 * (2 * STAGES + 4) + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_m = (M + BM - 1) / BM, n_n = N / BN, n_tiles = n_m * n_n, n_kb = K / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(full_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(tfull_bar(a), 1);
+      ptx::mbar_init(tempty_bar(a), 4);                     // one arrival per epilogue warp
+    }
+    abort_flag[0] = 0;
+    abort_flag[1] = 0;
+    ptx::fence_barrier_init();
+    ptx::fence_proxy_async();
+  }
+  if (warp == 2) {
+    ptx::tmem_alloc(ptx::smem_u32((const void*)tmem_slot), Cfg::TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      ptx::prefetch_tensormap(&tmap_a);
+      ptx::prefetch_tensormap(&tmap_w);
+      int it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const int m_blk = tile / n_n, n_blk = tile - m_blk * n_n;
+        for (int kb = 0; kb < n_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+          if (!ptx::mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+          ptx::mbar_expect_tx(full_bar(s), A_BYTES + Cfg::B_BYTES);
+          ptx::tma_load_2d(a_base + s * A_BYTES, &tmap_a, kb * BK, m_blk * BM, full_bar(s));
+          ptx::tma_load_2d(w_base + s * Cfg::B_BYTES, &tmap_w, kb * BK, n_blk * BN, full_bar(s));
+        }
+      }
+      if (!ok) {
+        *(volatile int*)status = ST_PRODUCER;
+        // let copies already issued land before the CTA's shared memory is released
+        for (int j = 1; j <= STAGES && j <= it; ++j) {
+          const int i2 = it - j;
+          ptx::mbar_wait(full_bar(i2 % STAGES), (uint32_t)(i2 / STAGES) & 1u, abort_flag + 1, 20000000LL);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = ptx::idesc_bf16_f32(BM, BN);
+      int it = 0, tile_i = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tile_i) {
+        const int acc = tile_i & 1;
+        const uint32_t acc_ph = (uint32_t)(tile_i >> 1) & 1u;
+        if (!ptx::mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < n_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+          if (!ptx::mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+          ptx::tc_fence_after();
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t da = ptx::smem_desc_k_sw128(a_base + s * A_BYTES + k * 32);
+            const uint64_t dw = ptx::smem_desc_k_sw128(w_base + s * Cfg::B_BYTES + k * 32);
+            ptx::umma_f16(d_tmem, da, dw, idesc, (kb | k) ? 1u : 0u);
+          }
+          ptx::umma_commit(empty_bar(s));                   // slot free once these MMAs have read it
+        }
+        if (ok) ptx::umma_commit(tfull_bar(acc));           // accumulator complete
+      }
+      if (!ok) *(volatile int*)status = ST_MMA;
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue (warps 2..5)
+    const int quarter = warp & 3;                           // TMEM lanes 32*quarter .. +31
+    int tile_i = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tile_i) {
+      const int m_blk = tile / n_n, n_blk = tile - m_blk * n_n;
+      const int acc = tile_i & 1;
+      const uint32_t acc_ph = (uint32_t)(tile_i >> 1) & 1u;
+      if (!ptx::mbar_wait(tfull_bar(acc), acc_ph, abort_flag)) { ok = false; break; }
+      ptx::tc_fence_after();
+      const int row = m_blk * BM + quarter * 32 + lane;
+      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        ptx::tmem_ld_32x32(t_row + (uint32_t)(c * 32), r);
+        ptx::tmem_ld_wait();
+        const int col = n_blk * BN + c * 32;
+        if (row < M) {
+          const float4* b4 = reinterpret_cast<const float4*>(bias + col);
+          if (EPI == 1) {
+            float4* o4 = reinterpret_cast<float4*>(reinterpret_cast<float*>(out_) + (size_t)row * N + col);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const float4 bv = __ldg(b4 + j);
+              float4 o = o4[j];
+              o.x += __uint_as_float(r[4 * j + 0]) + bv.x;
+              o.y += __uint_as_float(r[4 * j + 1]) + bv.y;
+              o.z += __uint_as_float(r[4 * j + 2]) + bv.z;
+              o.w += __uint_as_float(r[4 * j + 3]) + bv.w;
+              o4[j] = o;
+            }
+          } else {
+            uint4* o4 = reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(out_) + (size_t)row * N + col);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float4 b0 = __ldg(b4 + 2 * j), b1 = __ldg(b4 + 2 * j + 1);
+              float v0 = __uint_as_float(r[8 * j + 0]) + b0.x, v1 = __uint_as_float(r[8 * j + 1]) + b0.y;
+              float v2 = __uint_as_float(r[8 * j + 2]) + b0.z, v3 = __uint_as_float(r[8 * j + 3]) + b0.w;
+              float v4 = __uint_as_float(r[8 * j + 4]) + b1.x, v5 = __uint_as_float(r[8 * j + 5]) + b1.y;
+              float v6 = __uint_as_float(r[8 * j + 6]) + b1.z, v7 = __uint_as_float(r[8 * j + 7]) + b1.w;
+              if (EPI == 2) {
+                v0 = gelu_erf(v0); v1 = gelu_erf(v1); v2 = gelu_erf(v2); v3 = gelu_erf(v3);
+                v4 = gelu_erf(v4); v5 = gelu_erf(v5); v6 = gelu_erf(v6); v7 = gelu_erf(v7);
+              }
+              uint4 pk;
+              pk.x = pack_bf16x2(v0, v1); pk.y = pack_bf16x2(v2, v3);
+              pk.z = pack_bf16x2(v4, v5); pk.w = pack_bf16x2(v6, v7);
+              o4[j] = pk;
+            }
+          }
+        }
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+    }
+    if (!ok && lane == 0) *(volatile int*)status = ST_EPILOGUE;
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+  }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+// Row-major bf16 matrix [rows][cols] with row stride ld elements; box = 64 columns x box_rows rows.
+bool make_map_2d(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {ld * 2};
+  const cuuint32_t box[2] = {BK, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
+template <int BN, int EPI>
+cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tw, int M, int N, int K, const float* bias,
+                       void* out, int* status, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         GemmCfg<BN>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int n_tiles = ((M + BM - 1) / BM) * (N / BN);
+  const int grid = n_tiles < sm_count() ? n_tiles : sm_count();
+  gemm_tcgen05_kernel<BN, EPI><<<grid, kGemmThreads, GemmCfg<BN>::SMEM_BYTES, st>>>(ta, tw, M, N, K, bias, out, status);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+int gemm_tcgen05_pick_bn(int M, int N) {
+  const int n_m = (M + BM - 1) / BM, sms = sm_count();
+  if (N % 256) return 128;
+  const long t256 = (long)n_m * (N / 256), t128 = (long)n_m * (N / 128);
+  const double c256 = (double)((t256 + sms - 1) / sms) * 256.0;
+  const double c128 = (double)((t128 + sms - 1) / sms) * 128.0 * 1.08;   // smaller tiles re-read A more often
+  return c256 <= c128 ? 256 : 128;
+}
+
+cudaError_t launch_gemm_tcgen05(const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
+                                int epilogue, void* out, int* status, cudaStream_t st) {
+  if (M == 0) return cudaSuccess;
+  if (N % 128 || K % BK || lda % 8 || ((uintptr_t)a & 15) || ((uintptr_t)w & 15)) return cudaErrorInvalidValue;
+  const int bn = gemm_tcgen05_pick_bn(M, N);
+  CUtensorMap ta, tw;
+  if (!make_map_2d(&ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM)) return cudaErrorInvalidValue;
+  if (!make_map_2d(&tw, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)bn)) return cudaErrorInvalidValue;
+#define MARCHE_GEMM_CASE(BN_, EPI_) \
+  if (bn == BN_ && epilogue == EPI_) return launch_one<BN_, EPI_>(ta, tw, M, N, K, bias, out, status, st);
+  MARCHE_GEMM_CASE(256, 0) MARCHE_GEMM_CASE(256, 1) MARCHE_GEMM_CASE(256, 2)
+  MARCHE_GEMM_CASE(128, 0) MARCHE_GEMM_CASE(128, 1) MARCHE_GEMM_CASE(128, 2)
+#undef MARCHE_GEMM_CASE
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace marche

@@ -42,6 +42,12 @@ cudaError_t launch_topk(const float* partial, int H, float* scores, const uint8_
 cudaError_t launch_gemm_simt(bool bf16_t, const void* a, int lda, int M, const void* w, const float* bias,
                              int N, int K, int epilogue, void* out, cudaStream_t st);
 
+// K2 (bf16, tcgen05/TMEM fed by TMA).  N % 128 == 0, K % 64 == 0, lda % 8 == 0, 16-byte aligned
+// operands.  `status` is a device-visible int that bounded waits set when they give up.
+cudaError_t launch_gemm_tcgen05(const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
+                                int epilogue, void* out, int* status, cudaStream_t st);
+int gemm_tcgen05_pick_bn(int M, int N);
+
 // K3 (SIMT): attention of n queries per sample over all S cache rows.
 cudaError_t launch_attention_simt(bool bf16_t, const void* q, int ld_q, int B, int n, int S, int H, int dh,
                                   const void* cache_layer, const uint8_t* is_new, float* score_partial,

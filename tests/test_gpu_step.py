@@ -106,7 +106,8 @@ def test_invariants_untouched_rows_full_equivalence_reproducibility(dtype):
     # P5: rows outside A are byte-identical after a cache-aware step (sentinel in hidden_out)
     hidden2 = hidden.clone()
     for b in range(B):
-        hidden2[b, torch.as_tensor(A[b], dtype=torch.long)] += 0.5
+        # (not a constant shift: LayerNorm would remove it and leave K, V unchanged)
+        hidden2[b, torch.as_tensor(A[b], dtype=torch.long)] = torch.randn(A.shape[1], D, device="cuda")
     out = torch.full((B, S, D), 777.0, device="cuda")
     m.step(hidden2, cache, idx_dev(A), idx_dev(G), None, 0.1, out, refresh, ws)
     torch.cuda.synchronize()
