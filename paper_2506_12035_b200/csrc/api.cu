@@ -95,9 +95,14 @@ int do_linear(marche_ctx* ctx, const void* a, int lda, int M, const void* w, con
 int do_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void* cache_layer, const uint8_t* is_new,
                  float* partial, void* o, cudaStream_t st) {
   const marche_config& c = ctx->cfg;
-  MARCHE_TRY(launch_attention_simt(ctx->bf16, q, ld_q, c.batch, n, c.seq_len, c.n_heads, c.head_dim, cache_layer,
-                                   is_new, partial, o, st),
-             "attention");
+  const bool tc = ctx->bf16 && !ctx->force_simt && (c.head_dim == 64 || c.head_dim == 80) && ld_q % 2 == 0 &&
+                  ((uintptr_t)q & 3) == 0 && ((uintptr_t)cache_layer & 15) == 0;
+  if (tc)
+    MARCHE_TRY(launch_attention_mma(q, ld_q, c.batch, n, c.seq_len, c.n_heads, c.head_dim, cache_layer, is_new,
+                                    partial, o, ctx->status_dev, st), "attention_mma");
+  else
+    MARCHE_TRY(launch_attention_simt(ctx->bf16, q, ld_q, c.batch, n, c.seq_len, c.n_heads, c.head_dim, cache_layer,
+                                     is_new, partial, o, st), "attention");
   return MARCHE_OK;
 }
 

@@ -54,4 +54,10 @@ cudaError_t launch_attention_simt(bool bf16_t, const void* q, int ld_q, int B, i
                                   void* o, cudaStream_t st);
 size_t attention_simt_smem(int S, int dh);
 
+// K3 (bf16, TMA-staged K/V tiles, tensor-core QK^T and PV, fused score column sums).
+// head_dim 64 or 80; ld_q even; cache_layer 16-byte aligned.
+cudaError_t launch_attention_mma(const void* q, int ld_q, int B, int n, int S, int H, int dh,
+                                 const void* cache_layer, const uint8_t* is_new, float* score_partial, void* o,
+                                 int* status, cudaStream_t st);
+
 }  // namespace marche
