@@ -1,0 +1,359 @@
+#!/usr/bin/env python
+"""Benchmark of the MARche decoding hot path: 64-step synthetic MAR-L-shaped generation.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--config mar_l] [--ratio 0.1] [--blocks L] [--batch B] [--no-extras]
+
+One "step" of this benchmark is one whole T-step generation of a batch (B rows = B/2
+images with classifier-free-guidance pairs): a full step that fills the K/V cache and
+T-1 cache-aware steps, all through the C ABI of libmarche.  Only the transformer stack
+is timed; the sampler and the VAE are outside the hot path.  Rank 0 prints ONE JSON line.
+
+The path does not shard (one GPU holds a model replica and its own samples; there is no
+exchange step), so N > 1 runs N independent replicas and reports the aggregate
+("scaling": "weak").
+
+--impl reference times the CPU oracle (the deliberately plain NumPy restatement of the
+method) on a bounded sample of the same workload on this machine's host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+import synth
+
+# Fallback roofline denominators (an earlier measurement on this machine), used only when
+# MEASURED_PEAKS.json is absent.
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM traffic per launch of the dominant kernel classes from the committed ncu captures
+# (profiles/), bytes; None where no capture exists.
+NCU_TRAFFIC = {"gemm": None, "attention": None}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        self.lines = []
+        self.idx = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "power_w_max": float(max(power)), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- workload bookkeeping
+def schedule(cfg, ratio):
+    """Per step: (#G, nA, k) of the cache-aware generation (k selected at the step for the next)."""
+    counts = synth.mask_schedule(cfg.n_img, cfg.T)
+    want = int(np.floor(ratio * cfg.S + 0.5))
+    out, k_prev = [], 0
+    for t, g in enumerate(counts):
+        nxt = counts[t + 1] if t + 1 < cfg.T else 0
+        nA = cfg.S if t == 0 else g + counts[t - 1] + k_prev
+        k = min(want, cfg.S - g - nxt)
+        out.append((g, nA, k))
+        k_prev = k
+    return out
+
+
+def algorithmic_work(cfg, sched):
+    """Algorithmic flops / bytes per generation for each kernel class (bf16 operands, fp32 residual)."""
+    B, S, D, F, L, H = cfg.B, cfg.S, cfg.D, cfg.F, cfg.L, cfg.H
+    w = {"gemm_flops": 0.0, "attention_bytes": 0.0, "attention_flops": 0.0, "gather_layernorm_bytes": 0.0,
+         "scatter_kv_bytes": 0.0, "scatter_rows_bytes": 0.0, "topk_bytes": 0.0}
+    for g, nA, k in sched:
+        M = B * nA
+        w["gemm_flops"] += 2.0 * M * (4 * D * D + 2 * D * F) * L
+        w["attention_bytes"] += (2.0 * B * S * D * 2 + 2.0 * M * D * 2) * L + B * H * S * 4
+        w["attention_flops"] += 4.0 * B * nA * S * D * L
+        w["gather_layernorm_bytes"] += 2 * (M * D * 4 + M * D * 2) * L + M * D * 4
+        w["scatter_kv_bytes"] += 4.0 * M * D * 2 * L
+        w["scatter_rows_bytes"] += 2.0 * M * D * 4
+        w["topk_bytes"] += B * H * S * 4 + B * S * 5 + B * k * 4
+    return w
+
+
+# ----------------------------------------------------------------------------- reference arm (CPU oracle)
+def oracle_sample(cfg, ratio, n_cache_steps=2):
+    """Times the oracle on one CFG pair (2 of the B rows): 1 full step + n cache-aware steps,
+    and extrapolates to a T-step generation.  Returns (images_per_s, seconds_per_generation, dict)."""
+    from oracle import marche_oracle as orc
+    pair = cfg.replace(B=2)
+    blocks = synth.make_weights(cfg)
+    hidden = synth.make_hidden(cfg, batch=2)
+    orders = synth.generation_orders(cfg)
+    sets = [g[[0, cfg.B // 2]] if cfg.cfg_pairs else g[:2] for g in synth.new_token_sets(cfg, orders)]
+    kw = dict(n_heads=cfg.H, score_layer=cfg.score_layer, ln_eps=cfg.ln_eps)
+    cache = orc.KVCache(cfg.L, 2, cfg.S, cfg.D)
+    out = np.zeros_like(hidden)
+    t0 = time.perf_counter()
+    _, R = orc.full_step(blocks, hidden, cache, sets[0], sets[1], ratio, out, **kw)
+    t_full = time.perf_counter() - t0
+    t_steps = []
+    for t in range(1, 1 + n_cache_steps):
+        rows = synth.replacement_rows(cfg, t - 1, sets[t - 1].shape[1], batch=2)
+        for b in range(2):
+            hidden[b, sets[t - 1][b]] = rows[b]
+        A = orc.active_set(sets[t], sets[t - 1], R)
+        t0 = time.perf_counter()
+        _, R = orc.marche_step(blocks, hidden, cache, A, sets[t], sets[t + 1], ratio, out, **kw)
+        t_steps.append(time.perf_counter() - t0)
+    t_gen = t_full + (cfg.T - 1) * float(np.mean(t_steps))     # one image (its CFG pair), T steps
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    info = {"kind": "oracle", "cores": int(cores),
+            "sample": "one CFG pair (2 of %d rows): 1 full step (%.2f s) + %d cache-aware steps (%.2f s each), "
+                      "extrapolated to %d steps" % (cfg.B, t_full, n_cache_steps, float(np.mean(t_steps)), cfg.T)}
+    return 1.0 / t_gen, t_gen, info
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    for _ in range(args.steps):
+        ips, t_gen, info = oracle_sample(cfg, args.ratio)
+        vals.append((ips, t_gen))
+    ips = float(np.mean([v[0] for v in vals]))
+    t_gen = float(np.mean([v[1] for v in vals]))
+    info = dict(info, value=ips, unit="images/s")
+    line = {"impl": "reference", "metric": METRIC, "value": ips, "unit": "images/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_gen * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(cfg, args.ratio), "cpu_baseline": info,
+            "e2e": {"value": ips, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+METRIC = "images/s (64-step MAR-L-shaped, bs128)"
+
+
+def workload_config(cfg, ratio):
+    return {"workload": "%s: %d blocks, width %d, %d heads, MLP %d, %d tokens (%d image + %d buffer), batch %d "
+                        "(CFG-doubled), %d steps cosine schedule, refresh ratio %g; transformer stack only"
+                        % (cfg.name, cfg.L, cfg.D, cfg.H, cfg.F, cfg.S, cfg.n_img, cfg.n_buffer, cfg.B, cfg.T, ratio),
+            "config_name": cfg.name, "refresh_ratio": ratio, "l2": "working set (K/V cache + weights) exceeds L2",
+            "timed": "T-step generation per bench step"}
+
+
+# ----------------------------------------------------------------------------- our arm
+def run_ours(args, cfg):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2506_12035_b200.binding import Marche, upload_weights
+    from paper_2506_12035_b200.generation import Generation
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks, peak_kind = load_peaks()
+
+    ratio = args.ratio
+    blocks = synth.make_weights(cfg)
+    m = Marche.from_config(cfg, upload_weights(blocks, cfg.dtype))
+    del blocks
+    hidden0_np = synth.make_hidden(cfg)
+    sets = synth.new_token_sets(cfg, synth.generation_orders(cfg))
+    rows_np = [synth.replacement_rows(cfg, t, sets[t].shape[1]) for t in range(cfg.T)]
+    gen = Generation(m, sets, ratio, [torch.as_tensor(r).cuda() for r in rows_np])
+    hidden0 = torch.as_tensor(hidden0_np).cuda()
+    sched = schedule(cfg, ratio)
+    work = algorithmic_work(cfg, sched)
+    n_images = cfg.n_images
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, reps):
+        """max-over-ranks device time of `reps` calls of fn, in ms per call."""
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        barrier()
+        ms = torch.tensor([e0.elapsed_time(e1)], device="cuda")
+        if world > 1:
+            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+        return float(ms.item()) / reps
+
+    for _ in range(args.warmup):
+        gen.run(hidden0)
+    torch.cuda.synchronize()
+    clocks = ClockSampler(local)
+    clocks.start()
+    launches0 = m.launch_count()
+    ms_gen = timed(lambda: gen.run(hidden0), args.steps)
+    launches = m.launch_count() - launches0
+    clock_info = clocks.stop()
+    assert m.device_status() == 0, "a bounded device wait gave up"
+    value = world * n_images / (ms_gen * 1e-3)
+
+    line = {"metric": METRIC, "value": value, "unit": "images/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_gen, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": workload_config(cfg, ratio), "clocks": clock_info, "gpu_launches": int(launches),
+            "ms_per_decoding_step": ms_gen / cfg.T}
+
+    if not args.no_extras:
+        # ---- per-kernel-class device time of one more generation (events in front of every launch)
+        m.profile_begin()
+        gen.run(hidden0)
+        prof = m.profile_end()
+        gemm_ms = sum(prof[c][0] for c in ("gemm_qkv", "gemm_out_proj", "gemm_fc1_gelu", "gemm_fc2"))
+        gemm_n = sum(prof[c][1] for c in ("gemm_qkv", "gemm_out_proj", "gemm_fc1_gelu", "gemm_fc2"))
+        total_ms = sum(v[0] for v in prof.values())
+        kernels = []
+
+        def add(name, bound, amount, ms, n, peak, unit):
+            if n == 0 or ms <= 0:
+                return
+            ach = amount / (ms * 1e-3) / (1e12 if unit == "TFLOP/s" else 1e9)
+            kernels.append({"kernel": name, "bound": bound, "achieved": ach, "peak": peak, "unit": unit,
+                            "frac": ach / peak, "launches": n, "ms_per_generation": ms, "share": ms / total_ms})
+
+        add("gemm_tcgen05 (qkv, out, fc1, fc2)", "tensor", work["gemm_flops"], gemm_ms, gemm_n,
+            peaks["bf16_tflops_sustained"], "TFLOP/s")
+        add("attention", "hbm", work["attention_bytes"], prof["attention"][0], prof["attention"][1], peaks["hbm_gbs"], "GB/s")
+        add("gather_layernorm", "hbm", work["gather_layernorm_bytes"], prof["gather_layernorm"][0],
+            prof["gather_layernorm"][1], peaks["hbm_gbs"], "GB/s")
+        add("scatter_kv", "hbm", work["scatter_kv_bytes"], prof["scatter_kv"][0], prof["scatter_kv"][1], peaks["hbm_gbs"], "GB/s")
+        add("scatter_rows", "hbm", work["scatter_rows_bytes"], prof["scatter_rows"][0], prof["scatter_rows"][1],
+            peaks["hbm_gbs"], "GB/s")
+        add("topk", "hbm", work["topk_bytes"], prof["topk"][0], prof["topk"][1], peaks["hbm_gbs"], "GB/s")
+        kernels.sort(key=lambda k: -k["ms_per_generation"])
+        line["kernels"] = kernels
+        dom = kernels[0]
+        key = "gemm" if dom["bound"] == "tensor" else dom["kernel"]
+        line["roofline"] = {"kernel": dom["kernel"], "bound": dom["bound"], "achieved": dom["achieved"], "peak": dom["peak"],
+                            "unit": dom["unit"], "frac": dom["frac"], "traffic": NCU_TRAFFIC.get(key),
+                            "peak_source": "%s (%s)" % (peak_kind, "sustained bf16 GEMM" if dom["bound"] == "tensor" else "device copy"),
+                            "timing": "CUDA events in front of every launch of one generation of the timed workload"}
+
+        # ---- this build's own full-recompute path (full step at every decoding step)
+        gen.run(hidden0, mode="full")
+        ms_full = timed(lambda: gen.run(hidden0, mode="full"), 1)
+        line["full_recompute"] = {"value": world * n_images / (ms_full * 1e-3), "unit": "images/s", "ms_per_step": ms_full,
+                                  "speedup_cache_aware": ms_full / ms_gen}
+
+        # ---- end to end through marche_step_host: pinned host buffers, copies inside the timed region
+        gen.alloc_host_buffers(hidden0_np, rows_np, sets)
+        for _ in range(2):
+            h2d, d2h = gen.run_host()
+        ms_e2e = timed(lambda: gen.run_host(), args.steps)
+        line["e2e"] = {"value": world * n_images / (ms_e2e * 1e-3), "unit": "images/s", "h2d_bytes_per_step": int(h2d),
+                       "d2h_bytes_per_step": int(d2h), "ms_per_step": ms_e2e}
+        assert m.device_status() == 0
+
+        # ---- CPU oracle on a bounded sample (rank 0, N = 1 only)
+        if world == 1 and not args.no_cpu_baseline:
+            ips, _, info = oracle_sample(cfg, ratio)
+            line["cpu_baseline"] = dict(info, value=ips, unit="images/s")
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="mar_l", choices=list(synth.CONFIGS))
+    ap.add_argument("--ratio", type=float, default=0.10)
+    ap.add_argument("--blocks", type=int, default=0, help="override the depth (profiling captures only)")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling captures only)")
+    ap.add_argument("--tsteps", type=int, default=0, help="override the decoding steps (profiling captures only)")
+    ap.add_argument("--no-extras", action="store_true", help="only the timed region (for ncu launch lists)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = synth.CONFIGS[args.config]
+    if args.blocks:
+        cfg = cfg.replace(L=args.blocks, E=min(cfg.E, max(0, args.blocks - 2)))
+    if args.batch:
+        cfg = cfg.replace(B=args.batch)
+    if args.tsteps:
+        cfg = cfg.replace(T=args.tsteps)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

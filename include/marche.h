@@ -68,6 +68,14 @@ enum {
   MARCHE_EPI_BIAS_GELU = 2      /* out T[M][N]      = GELU_erf(acc + bias)                */
 };
 
+/* Kernel classes of marche_profile_end / marche_kernel_class_name. */
+enum {
+  MARCHE_KC_FLAGS = 0, MARCHE_KC_GATHER_LN = 1, MARCHE_KC_GEMM_QKV = 2, MARCHE_KC_SCATTER_KV = 3,
+  MARCHE_KC_ATTENTION = 4, MARCHE_KC_GEMM_O = 5, MARCHE_KC_GEMM_FC1 = 6, MARCHE_KC_GEMM_FC2 = 7,
+  MARCHE_KC_SCATTER_ROWS = 8, MARCHE_KC_TOPK = 9, MARCHE_KC_OTHER = 10,
+  MARCHE_N_KERNEL_CLASSES = 11
+};
+
 typedef struct {
   int32_t n_blocks;     /* L                                                              */
   int32_t n_enc_blocks; /* E; only used for the default score layer                       */
@@ -194,6 +202,38 @@ int marche_build_active(marche_ctx* ctx, const int32_t* new_idx, int n_new,
 int marche_scatter_rows(marche_ctx* ctx, const float* rows, const int32_t* idx, int n,
                         float* dst, marche_stream stream);
 
+/* Inverse of marche_scatter_rows: rows_out[b][j][:] = src[b][idx[b][j]][:], float
+ * [B][S][D] -> float [B][n][D]: the stack outputs z_i of the tokens being generated,
+ * which are all that the sampler consumes (Eq. 3). */
+int marche_gather_rows(marche_ctx* ctx, const float* src, const int32_t* idx, int n, float* rows_out,
+                       marche_stream stream);
+
+/* One decoding step driven from HOST buffers (a sampler that lives on the host): copies
+ * this step's inputs to the device, runs the step, copies its results back, all on
+ * `stream` (asynchronous when the host buffers are pinned; synchronise before reading).
+ *   full            non-zero: marche_full_step (first step); zero: cache-aware step with
+ *                   A = new | prev | refresh_in (Algorithm 1 line 4)
+ *   hidden          i/o device float [B][S][D], the stack input kept on the device; rows
+ *                   prev_idx are first overwritten with h_prev_rows (the tokens sampled
+ *                   after the previous step, Eq. 3-4)
+ *   h_prev_rows     host float [B][n_prev][D];  h_prev_idx host int32 [B][n_prev]
+ *   h_new_idx       host int32 [B][n_new] (G);  h_excl_idx host int32 [B][n_excl] or NULL
+ *   refresh_in      device int32 [B][n_refresh_in]: the previous call's refresh_out
+ *   refresh_out     device int32, room for B*floor(ratio*S+1/2) entries (the next call's
+ *                   refresh_in; use two buffers alternately)
+ *   h_out_rows      host float [B][n_new][D] or NULL: hidden_out rows of new_idx
+ *   h_refresh_out   host int32 [B][K] or NULL;  n_refresh host int, receives K
+ *   staging         device scratch of marche_staging_bytes(ctx, max_new), 256-byte aligned,
+ *                   where max_new bounds n_prev, n_new and n_excl
+ * Other arguments and errors as for marche_step / marche_full_step. */
+size_t marche_staging_bytes(const marche_ctx* ctx, int max_new);
+int marche_step_host(marche_ctx* ctx, int full, float* hidden, void* kv_cache, const float* h_prev_rows,
+                     const int32_t* h_prev_idx, int n_prev, const int32_t* h_new_idx, int n_new,
+                     const int32_t* h_excl_idx, int n_excl, const int32_t* refresh_in, int n_refresh_in,
+                     float refresh_ratio, float* hidden_out, int32_t* refresh_out, float* h_out_rows,
+                     int32_t* h_refresh_out, int* n_refresh, int max_new, void* staging, size_t staging_bytes,
+                     void* workspace, size_t workspace_bytes, marche_stream stream);
+
 /* Checks index sets on the device (range, uniqueness within a sample, new_idx a
  * subset of active_idx, exclude_idx disjoint from new_idx) and waits for the
  * result: MARCHE_OK or MARCHE_EINDEX.  Synchronous.  active_idx may be NULL
@@ -249,6 +289,16 @@ const char* marche_last_error(const marche_ctx* ctx);
  * invalid).  It lives in pinned host memory owned by the context; synchronise
  * the stream before reading it. */
 int marche_device_status(const marche_ctx* ctx);
+/* Number of kernels this context has launched so far. */
+unsigned long long marche_launch_count(const marche_ctx* ctx);
+/* Per-kernel-class device time of the calls made between marche_profile_begin and
+ * marche_profile_end: while profiling, a CUDA event is recorded on the stream in front
+ * of every launch, and the time up to the next event (the kernel plus the gap before its
+ * successor) is charged to the launch's class.  marche_profile_end synchronises the
+ * stream and fills two host arrays of MARCHE_N_KERNEL_CLASSES entries. */
+int marche_profile_begin(marche_ctx* ctx);
+int marche_profile_end(marche_ctx* ctx, marche_stream stream, float* ms_per_class, int* launches_per_class);
+const char* marche_kernel_class_name(int kernel_class);
 void marche_clear_device_status(marche_ctx* ctx);
 
 #ifdef __cplusplus

@@ -58,6 +58,14 @@ _SIGNATURES = {
     "marche_linear": (C.c_int, [_vp, _vp, _i, _i, _vp, _vp, _i, _i, _i, _vp, _vp]),
     "marche_scatter_kv": (C.c_int, [_vp, _vp, _vp, _i, _vp, _i, _vp, _vp]),
     "marche_attention": (C.c_int, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
+    "marche_gather_rows": (C.c_int, [_vp, _vp, _vp, _i, _vp, _vp]),
+    "marche_staging_bytes": (_sz, [_vp, _i]),
+    "marche_step_host": (C.c_int, [_vp, _i, _vp, _vp, _vp, _vp, _i, _vp, _i, _vp, _i, _vp, _i, _f, _vp, _vp, _vp, _vp,
+                                   C.POINTER(C.c_int), _i, _vp, _sz, _vp, _sz, _vp]),
+    "marche_launch_count": (C.c_ulonglong, [_vp]),
+    "marche_profile_begin": (C.c_int, [_vp]),
+    "marche_profile_end": (C.c_int, [_vp, _vp, C.POINTER(C.c_float), C.POINTER(C.c_int)]),
+    "marche_kernel_class_name": (C.c_char_p, [C.c_int]),
     "marche_strerror": (C.c_char_p, [C.c_int]),
     "marche_last_error": (C.c_char_p, [_vp]),
     "marche_device_status": (C.c_int, [_vp]),
@@ -239,6 +247,42 @@ class Marche:
     def attention(self, q, ld_q, n, cache_layer, is_new, score_partial, o, stream=None):
         self._check(self.lib.marche_attention(self.h, q.data_ptr(), ld_q, n, _ptr(cache_layer), _ptr(is_new),
                                               _ptr(score_partial), _ptr(o), _stream(stream)))
+
+    def gather_rows(self, src, idx, rows_out, stream=None):
+        self._check(self.lib.marche_gather_rows(self.h, _ptr(src), _ptr(idx), idx.shape[1], _ptr(rows_out),
+                                                _stream(stream)))
+
+    def staging_bytes(self, max_new: int) -> int:
+        return self.lib.marche_staging_bytes(self.h, max_new)
+
+    def step_host(self, full, hidden, kv_cache, h_prev_rows, h_prev_idx, h_new_idx, h_excl_idx, refresh_in,
+                  n_refresh_in, refresh_ratio, hidden_out, refresh_out, h_out_rows, h_refresh_out, max_new, staging,
+                  workspace, stream=None) -> int:
+        """Host tensors (h_*) are CPU tensors, pinned for asynchronous copies; the rest are CUDA tensors."""
+        def hp(t):
+            return None if t is None else t.data_ptr()
+        k = C.c_int(0)
+        self._check(self.lib.marche_step_host(
+            self.h, 1 if full else 0, _ptr(hidden), _ptr(kv_cache), hp(h_prev_rows), hp(h_prev_idx),
+            0 if h_prev_idx is None else h_prev_idx.shape[1], hp(h_new_idx), 0 if h_new_idx is None else h_new_idx.shape[1],
+            hp(h_excl_idx), 0 if h_excl_idx is None else h_excl_idx.shape[1], _ptr(refresh_in) if n_refresh_in else None,
+            n_refresh_in, refresh_ratio, _ptr(hidden_out), _ptr(refresh_out), hp(h_out_rows), hp(h_refresh_out),
+            C.byref(k), max_new, _ptr(staging), staging.numel(), _ptr(workspace), workspace.numel(), _stream(stream)))
+        return k.value
+
+    def launch_count(self) -> int:
+        return int(self.lib.marche_launch_count(self.h))
+
+    def profile_begin(self):
+        self._check(self.lib.marche_profile_begin(self.h))
+
+    def profile_end(self, stream=None):
+        """-> {class name: (milliseconds, launches)} for the calls since profile_begin."""
+        n = 11
+        ms = (C.c_float * n)()
+        cnt = (C.c_int * n)()
+        self._check(self.lib.marche_profile_end(self.h, _stream(stream), ms, cnt))
+        return {self.lib.marche_kernel_class_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n)}
 
     def device_status(self) -> int:
         return self.lib.marche_device_status(self.h)

@@ -37,6 +37,11 @@ struct marche_ctx {
   int* status_host = nullptr;                         // pinned, mapped
   int* status_dev = nullptr;
   std::string last_error;
+  // launch accounting and optional per-kernel-class timing
+  unsigned long long launches = 0;
+  bool profiling = false;
+  std::vector<cudaEvent_t> events;     // pool, reused between profile runs
+  std::vector<int> event_class;        // class of the launch that follows event i
 };
 
 namespace {
@@ -76,13 +81,29 @@ int cuda_fail(marche_ctx* c, cudaError_t e, const char* what) {
     if (e__ != cudaSuccess) return cuda_fail(ctx, e__, what); \
   } while (0)
 
+// Counts a launch and, while profiling, records an event in front of it.  The time from
+// this event to the next one (kernel plus the gap before its successor) is charged to `cls`.
+void mark(marche_ctx* ctx, int cls, cudaStream_t st) {
+  ++ctx->launches;
+  if (!ctx->profiling) return;
+  const size_t i = ctx->event_class.size();
+  if (i >= ctx->events.size()) {
+    cudaEvent_t e;
+    if (cudaEventCreate(&e) != cudaSuccess) return;
+    ctx->events.push_back(e);
+  }
+  cudaEventRecord(ctx->events[i], st);
+  ctx->event_class.push_back(cls);
+}
+
 int refresh_count(float ratio, int S, int n_cand) {
   const int want = (int)std::floor((double)ratio * (double)S + 0.5);
   return want < n_cand ? (want < 0 ? 0 : want) : n_cand;
 }
 
-int do_linear(marche_ctx* ctx, const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
+int do_linear(marche_ctx* ctx, int cls, const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
               int epi, void* out, cudaStream_t st) {
+  if (M > 0) mark(ctx, cls, st);
   const bool tc = ctx->bf16 && !ctx->force_simt && N % 128 == 0 && K % 64 == 0 && lda % 8 == 0 &&
                   (((uintptr_t)a | (uintptr_t)w | (uintptr_t)out) & 15) == 0;
   if (tc)
@@ -95,6 +116,7 @@ int do_linear(marche_ctx* ctx, const void* a, int lda, int M, const void* w, con
 int do_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void* cache_layer, const uint8_t* is_new,
                  float* partial, void* o, cudaStream_t st) {
   const marche_config& c = ctx->cfg;
+  if (n > 0) mark(ctx, MARCHE_KC_ATTENTION, st);
   const bool tc = ctx->bf16 && !ctx->force_simt && (c.head_dim == 64 || c.head_dim == 80) && ld_q % 2 == 0 &&
                   ((uintptr_t)q & 3) == 0 && ((uintptr_t)cache_layer & 15) == 0;
   if (tc)
@@ -136,32 +158,38 @@ int run_stack(marche_ctx* ctx, const float* hidden, void* kv_cache, const int32_
   const size_t eb = ctx->eb;
   const size_t layer_bytes = (size_t)2 * B * S * D * eb;
 
+  mark(ctx, MARCHE_KC_FLAGS, st);
   MARCHE_TRY(launch_step_flags(active_idx, nA, new_idx, n_new, excl_idx, n_excl, B, S, is_new, cand, st), "flags");
   for (int l = 0; l < L; ++l) {
     const marche_block_weights& bw = ctx->blocks[l];
     char* cache_l = (char*)kv_cache + (size_t)l * layer_bytes;
+    mark(ctx, MARCHE_KC_GATHER_LN, st);
     if (l == 0)
       MARCHE_TRY(launch_gather_layernorm(ctx->bf16, hidden, S, active_idx, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
                                          x, u, st), "gather_layernorm");
     else
       MARCHE_TRY(launch_gather_layernorm(ctx->bf16, x, nA, nullptr, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
                                          nullptr, u, st), "layernorm1");
-    int rc = do_linear(ctx, u, D, M, bw.w_qkv, bw.b_qkv, 3 * D, D, MARCHE_EPI_BIAS, qkv, st);
+    int rc = do_linear(ctx, MARCHE_KC_GEMM_QKV, u, D, M, bw.w_qkv, bw.b_qkv, 3 * D, D, MARCHE_EPI_BIAS, qkv, st);
     if (rc) return rc;
+    mark(ctx, MARCHE_KC_SCATTER_KV, st);
     MARCHE_TRY(launch_scatter_kv(ctx->bf16, qkv + (size_t)D * eb, qkv + (size_t)2 * D * eb, 3 * D, active_idx, B, nA,
                                  S, D, cache_l, st), "scatter_kv");
     rc = do_attention(ctx, qkv, 3 * D, nA, cache_l, l == ctx->score_layer ? is_new : nullptr, partial, o, st);
     if (rc) return rc;
-    rc = do_linear(ctx, o, D, M, bw.w_o, bw.b_o, D, D, MARCHE_EPI_BIAS_RESIDUAL, x, st);
+    rc = do_linear(ctx, MARCHE_KC_GEMM_O, o, D, M, bw.w_o, bw.b_o, D, D, MARCHE_EPI_BIAS_RESIDUAL, x, st);
     if (rc) return rc;
+    mark(ctx, MARCHE_KC_GATHER_LN, st);
     MARCHE_TRY(launch_gather_layernorm(ctx->bf16, x, nA, nullptr, B, nA, D, bw.ln2_g, bw.ln2_b, ctx->eps, nullptr,
                                        u, st), "layernorm2");
-    rc = do_linear(ctx, u, D, M, bw.w_fc1, bw.b_fc1, F, D, MARCHE_EPI_BIAS_GELU, g, st);
+    rc = do_linear(ctx, MARCHE_KC_GEMM_FC1, u, D, M, bw.w_fc1, bw.b_fc1, F, D, MARCHE_EPI_BIAS_GELU, g, st);
     if (rc) return rc;
-    rc = do_linear(ctx, g, F, M, bw.w_fc2, bw.b_fc2, D, F, MARCHE_EPI_BIAS_RESIDUAL, x, st);
+    rc = do_linear(ctx, MARCHE_KC_GEMM_FC2, g, F, M, bw.w_fc2, bw.b_fc2, D, F, MARCHE_EPI_BIAS_RESIDUAL, x, st);
     if (rc) return rc;
   }
+  mark(ctx, MARCHE_KC_SCATTER_ROWS, st);
   MARCHE_TRY(launch_scatter_rows(x, active_idx, B, nA, S, D, hidden_out, st), "scatter_rows");
+  mark(ctx, MARCHE_KC_TOPK, st);
   MARCHE_TRY(launch_topk(partial, H, scores, cand, B, S, k, refresh_idx, st), "topk");
   return MARCHE_OK;
 }
@@ -218,6 +246,7 @@ int marche_create(const marche_config* cfg, const marche_block_weights* blocks, 
 void marche_destroy(marche_ctx* ctx) {
   if (!ctx) return;
   if (ctx->status_host) cudaFreeHost(ctx->status_host);
+  for (cudaEvent_t e : ctx->events) cudaEventDestroy(e);
   delete ctx;
 }
 
@@ -277,8 +306,10 @@ int marche_select_refresh(marche_ctx* ctx, const float* scores, const int32_t* n
   if (k == 0) return MARCHE_OK;
   if (!refresh_idx) return MARCHE_EINVAL;
   cudaStream_t st = (cudaStream_t)stream;
+  mark(ctx, MARCHE_KC_FLAGS, st);
   MARCHE_TRY(launch_step_flags(nullptr, 0, new_idx, n_new, exclude_idx, n_excl, B, S, nullptr, (uint8_t*)mask_scratch,
                                st), "flags");
+  mark(ctx, MARCHE_KC_TOPK, st);
   MARCHE_TRY(launch_topk(nullptr, 0, const_cast<float*>(scores), (const uint8_t*)mask_scratch, B, S, k, refresh_idx,
                          st), "topk");
   return MARCHE_OK;
@@ -297,6 +328,7 @@ int marche_build_active(marche_ctx* ctx, const int32_t* new_idx, int n_new, cons
   if (!ctx || !active_idx || n_new < 0 || n_prev < 0 || n_refresh < 0) return MARCHE_EINVAL;
   if ((n_new && !new_idx) || (n_prev && !prev_idx) || (n_refresh && !refresh_idx)) return MARCHE_EINVAL;
   if (n_new + n_prev + n_refresh > ctx->cfg.seq_len) return MARCHE_EINVAL;
+  mark(ctx, MARCHE_KC_OTHER, (cudaStream_t)stream);
   MARCHE_TRY(launch_build_active(new_idx, n_new, prev_idx, n_prev, refresh_idx, n_refresh, ctx->cfg.batch, active_idx,
                                  (cudaStream_t)stream), "build_active");
   return MARCHE_OK;
@@ -305,6 +337,8 @@ int marche_build_active(marche_ctx* ctx, const int32_t* new_idx, int n_new, cons
 int marche_scatter_rows(marche_ctx* ctx, const float* rows, const int32_t* idx, int n, float* dst,
                         marche_stream stream) {
   if (!ctx || !rows || !dst || n < 0 || n > ctx->cfg.seq_len || (n && !idx)) return MARCHE_EINVAL;
+  if (n == 0) return MARCHE_OK;
+  mark(ctx, MARCHE_KC_SCATTER_ROWS, (cudaStream_t)stream);
   MARCHE_TRY(launch_scatter_rows(rows, idx, ctx->cfg.batch, n, ctx->cfg.seq_len, ctx->cfg.width, dst,
                                  (cudaStream_t)stream), "scatter_rows");
   return MARCHE_OK;
@@ -330,6 +364,7 @@ int marche_gather_layernorm(marche_ctx* ctx, const float* src, int src_rows, con
                             marche_stream stream) {
   if (!ctx || !src || !gamma || !beta || !u_out || n < 0 || src_rows < 1) return MARCHE_EINVAL;
   if (!idx && n > src_rows) return MARCHE_EINVAL;
+  mark(ctx, MARCHE_KC_GATHER_LN, (cudaStream_t)stream);
   MARCHE_TRY(launch_gather_layernorm(ctx->bf16, src, src_rows, idx, ctx->cfg.batch, n, ctx->cfg.width, gamma, beta,
                                      ctx->eps, x_out, u_out, (cudaStream_t)stream), "gather_layernorm");
   return MARCHE_OK;
@@ -340,7 +375,7 @@ int marche_linear(marche_ctx* ctx, const void* a, int lda, int M, const void* w,
   if (!ctx || !a || !w || !bias || !out || M < 0 || N < 1 || K < 1 || lda < K) return MARCHE_EINVAL;
   if (epilogue < 0 || epilogue > 2) return MARCHE_EINVAL;
   if (ctx->bf16 ? (N % 128 || K % 64 || lda % 8) : (N % 64 || K % 16 || lda % 4)) return MARCHE_ESHAPE;
-  return do_linear(ctx, a, lda, M, w, bias, N, K, epilogue, out, (cudaStream_t)stream);
+  return do_linear(ctx, MARCHE_KC_OTHER, a, lda, M, w, bias, N, K, epilogue, out, (cudaStream_t)stream);
 }
 
 int marche_scatter_kv(marche_ctx* ctx, const void* k, const void* v, int ld_kv, const int32_t* idx, int n,
@@ -348,6 +383,7 @@ int marche_scatter_kv(marche_ctx* ctx, const void* k, const void* v, int ld_kv, 
   if (!ctx || !k || !v || !cache_layer || n < 0 || n > ctx->cfg.seq_len || ld_kv < ctx->cfg.width)
     return MARCHE_EINVAL;
   if (!idx && n != ctx->cfg.seq_len) return MARCHE_EINVAL;
+  mark(ctx, MARCHE_KC_SCATTER_KV, (cudaStream_t)stream);
   MARCHE_TRY(launch_scatter_kv(ctx->bf16, k, v, ld_kv, idx, ctx->cfg.batch, n, ctx->cfg.seq_len, ctx->cfg.width,
                                cache_layer, (cudaStream_t)stream), "scatter_kv");
   return MARCHE_OK;
@@ -359,6 +395,115 @@ int marche_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void
     return MARCHE_EINVAL;
   if (is_new && !score_partial) return MARCHE_EINVAL;
   return do_attention(ctx, q, ld_q, n, cache_layer, is_new, score_partial, o, (cudaStream_t)stream);
+}
+
+int marche_gather_rows(marche_ctx* ctx, const float* src, const int32_t* idx, int n, float* rows_out,
+                       marche_stream stream) {
+  if (!ctx || !src || !rows_out || n < 0 || n > ctx->cfg.seq_len || (n && !idx)) return MARCHE_EINVAL;
+  if (n == 0) return MARCHE_OK;
+  mark(ctx, MARCHE_KC_OTHER, (cudaStream_t)stream);
+  MARCHE_TRY(launch_gather_rows(src, idx, ctx->cfg.batch, n, ctx->cfg.seq_len, ctx->cfg.width, rows_out,
+                                (cudaStream_t)stream), "gather_rows");
+  return MARCHE_OK;
+}
+
+size_t marche_staging_bytes(const marche_ctx* ctx, int max_new) {
+  if (!ctx || max_new < 0 || max_new > ctx->cfg.seq_len) return 0;
+  const size_t B = ctx->cfg.batch, S = ctx->cfg.seq_len, D = ctx->cfg.width, n = max_new;
+  return 2 * align256(B * n * D * sizeof(float)) + 3 * align256(B * n * sizeof(int32_t)) +
+         align256(B * S * sizeof(int32_t));
+}
+
+int marche_step_host(marche_ctx* ctx, int full, float* hidden, void* kv_cache, const float* h_prev_rows,
+                     const int32_t* h_prev_idx, int n_prev, const int32_t* h_new_idx, int n_new,
+                     const int32_t* h_excl_idx, int n_excl, const int32_t* refresh_in, int n_refresh_in,
+                     float refresh_ratio, float* hidden_out, int32_t* refresh_out, float* h_out_rows,
+                     int32_t* h_refresh_out, int* n_refresh, int max_new, void* staging, size_t staging_bytes,
+                     void* workspace, size_t workspace_bytes, marche_stream stream) {
+  if (!ctx || !hidden || !staging || !refresh_out || n_prev < 0 || n_new < 0 || n_excl < 0 || n_refresh_in < 0)
+    return MARCHE_EINVAL;
+  if (n_prev > max_new || n_new > max_new || n_excl > max_new) return MARCHE_EINVAL;
+  if ((n_prev && (!h_prev_rows || !h_prev_idx)) || (n_new && !h_new_idx) || (n_excl && !h_excl_idx) ||
+      (n_refresh_in && !refresh_in))
+    return MARCHE_EINVAL;
+  if (((uintptr_t)staging & 255) != 0) return MARCHE_EINVAL;
+  if (staging_bytes < marche_staging_bytes(ctx, max_new)) return MARCHE_EWORKSPACE;
+  const size_t B = ctx->cfg.batch, S = ctx->cfg.seq_len, D = ctx->cfg.width, mn = max_new;
+  cudaStream_t st = (cudaStream_t)stream;
+  char* p = (char*)staging;
+  float* d_prev_rows = (float*)p;  p += align256(B * mn * D * sizeof(float));
+  float* d_out_rows = (float*)p;   p += align256(B * mn * D * sizeof(float));
+  int32_t* d_prev_idx = (int32_t*)p; p += align256(B * mn * sizeof(int32_t));
+  int32_t* d_new_idx = (int32_t*)p;  p += align256(B * mn * sizeof(int32_t));
+  int32_t* d_excl_idx = (int32_t*)p; p += align256(B * mn * sizeof(int32_t));
+  int32_t* d_active = (int32_t*)p;
+  if (n_prev) {
+    MARCHE_TRY(cudaMemcpyAsync(d_prev_rows, h_prev_rows, B * n_prev * D * sizeof(float), cudaMemcpyHostToDevice, st), "h2d");
+    MARCHE_TRY(cudaMemcpyAsync(d_prev_idx, h_prev_idx, B * n_prev * sizeof(int32_t), cudaMemcpyHostToDevice, st), "h2d");
+  }
+  if (n_new)
+    MARCHE_TRY(cudaMemcpyAsync(d_new_idx, h_new_idx, B * n_new * sizeof(int32_t), cudaMemcpyHostToDevice, st), "h2d");
+  if (n_excl)
+    MARCHE_TRY(cudaMemcpyAsync(d_excl_idx, h_excl_idx, B * n_excl * sizeof(int32_t), cudaMemcpyHostToDevice, st), "h2d");
+  int rc = marche_scatter_rows(ctx, d_prev_rows, d_prev_idx, n_prev, hidden, stream);
+  if (rc) return rc;
+  int k = 0;
+  if (full) {
+    rc = marche_full_step(ctx, hidden, kv_cache, d_new_idx, n_new, n_excl ? d_excl_idx : nullptr, n_excl,
+                          refresh_ratio, hidden_out, refresh_out, &k, workspace, workspace_bytes, stream);
+  } else {
+    const int nA = n_new + n_prev + n_refresh_in;
+    rc = marche_build_active(ctx, d_new_idx, n_new, d_prev_idx, n_prev, refresh_in, n_refresh_in, d_active, stream);
+    if (rc) return rc;
+    rc = marche_step(ctx, hidden, kv_cache, d_active, nA, d_new_idx, n_new, n_excl ? d_excl_idx : nullptr, n_excl,
+                     refresh_ratio, hidden_out, refresh_out, &k, workspace, workspace_bytes, stream);
+  }
+  if (rc) return rc;
+  if (n_refresh) *n_refresh = k;
+  if (h_out_rows && n_new) {
+    rc = marche_gather_rows(ctx, hidden_out, d_new_idx, n_new, d_out_rows, stream);
+    if (rc) return rc;
+    MARCHE_TRY(cudaMemcpyAsync(h_out_rows, d_out_rows, B * n_new * D * sizeof(float), cudaMemcpyDeviceToHost, st), "d2h");
+  }
+  if (h_refresh_out && k)
+    MARCHE_TRY(cudaMemcpyAsync(h_refresh_out, refresh_out, B * k * sizeof(int32_t), cudaMemcpyDeviceToHost, st), "d2h");
+  return MARCHE_OK;
+}
+
+unsigned long long marche_launch_count(const marche_ctx* ctx) { return ctx ? ctx->launches : 0ull; }
+
+int marche_profile_begin(marche_ctx* ctx) {
+  if (!ctx) return MARCHE_EINVAL;
+  ctx->event_class.clear();
+  ctx->profiling = true;
+  return MARCHE_OK;
+}
+
+int marche_profile_end(marche_ctx* ctx, marche_stream stream, float* ms_per_class, int* launches_per_class) {
+  if (!ctx || !ms_per_class || !launches_per_class) return MARCHE_EINVAL;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t n = ctx->event_class.size();
+  mark(ctx, MARCHE_KC_OTHER, st);              // closing event
+  --ctx->launches;
+  ctx->profiling = false;
+  for (int c = 0; c < MARCHE_N_KERNEL_CLASSES; ++c) { ms_per_class[c] = 0.f; launches_per_class[c] = 0; }
+  if (ctx->event_class.size() != n + 1) { ctx->event_class.clear(); return MARCHE_ECUDA; }
+  MARCHE_TRY(cudaStreamSynchronize(st), "sync");
+  for (size_t i = 0; i < n; ++i) {
+    float ms = 0.f;
+    MARCHE_TRY(cudaEventElapsedTime(&ms, ctx->events[i], ctx->events[i + 1]), "elapsed");
+    ms_per_class[ctx->event_class[i]] += ms;
+    ++launches_per_class[ctx->event_class[i]];
+  }
+  ctx->event_class.clear();
+  return MARCHE_OK;
+}
+
+const char* marche_kernel_class_name(int cls) {
+  static const char* names[MARCHE_N_KERNEL_CLASSES] = {
+      "step_flags", "gather_layernorm", "gemm_qkv", "scatter_kv", "attention", "gemm_out_proj",
+      "gemm_fc1_gelu", "gemm_fc2", "scatter_rows", "topk", "other"};
+  return (cls >= 0 && cls < MARCHE_N_KERNEL_CLASSES) ? names[cls] : "?";
 }
 
 const char* marche_strerror(int code) {

@@ -44,6 +44,18 @@ scatter_rows_kernel(const float4* __restrict__ rows, const int32_t* __restrict__
   for (int c = lane; c < row_vecs; c += 32) d[c] = __ldg(src + c);
 }
 
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const float4* __restrict__ src, const int32_t* __restrict__ idx, int n, int S, int row_vecs,
+                   long total_rows, float4* __restrict__ out) {
+  const long r = (long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (r >= total_rows) return;
+  const int b = (int)(r / n);
+  const float4* s = src + ((long)b * S + idx[r]) * row_vecs;
+  float4* d = out + r * row_vecs;
+  for (int c = lane; c < row_vecs; c += 32) d[c] = __ldg(s + c);
+}
+
 // One CTA per sample.  mark bit0 = generating token, bit1 = excluded token.
 __global__ void __launch_bounds__(256)
 step_flags_kernel(const int32_t* __restrict__ active_idx, int n_active, const int32_t* __restrict__ new_idx,
@@ -129,6 +141,16 @@ cudaError_t launch_scatter_rows(const float* rows, const int32_t* idx, int B, in
   if (total == 0) return cudaSuccess;
   scatter_rows_kernel<<<(unsigned)((total + 7) / 8), 256, 0, st>>>((const float4*)rows, idx, n, S, D / 4, total,
                                                                   (float4*)dst);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gather_rows(const float* src, const int32_t* idx, int B, int n, int S, int D, float* out,
+                               cudaStream_t st) {
+  if (D % 4) return cudaErrorInvalidValue;
+  const long total = (long)B * n;
+  if (total == 0) return cudaSuccess;
+  gather_rows_kernel<<<(unsigned)((total + 7) / 8), 256, 0, st>>>((const float4*)src, idx, n, S, D / 4, total,
+                                                                 (float4*)out);
   return cudaGetLastError();
 }
 

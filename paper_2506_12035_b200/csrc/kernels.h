@@ -21,6 +21,10 @@ cudaError_t launch_scatter_kv(bool bf16_t, const void* k, const void* v, int ld_
 cudaError_t launch_scatter_rows(const float* rows, const int32_t* idx, int B, int n, int S, int D,
                                 float* dst, cudaStream_t st);
 
+// fp32 row gather out[b][j] = src[b][idx[b][j]].
+cudaError_t launch_gather_rows(const float* src, const int32_t* idx, int B, int n, int S, int D, float* out,
+                               cudaStream_t st);
+
 // a0 prologue: is_new[b][j] (may be NULL with n_active = 0) and the candidate mask cand[b][t].
 cudaError_t launch_step_flags(const int32_t* active_idx, int n_active, const int32_t* new_idx, int n_new,
                               const int32_t* excl_idx, int n_excl, int B, int S, uint8_t* is_new,

@@ -75,3 +75,42 @@ class Generation:
             m.scatter_rows(self.rows[t], G, self.hidden, stream)
             k_prev = k
         return log
+
+    # ------------------------------------------------------------------ host-driven loop
+    def alloc_host_buffers(self, hidden0, rows_np, sets_np):
+        """Pinned host buffers for run_host: the stack input, per step the sampled rows and
+        index sets (inputs) and the output rows / refresh indices (results)."""
+        pin = lambda a: torch.as_tensor(a).contiguous().pin_memory()
+        B, S, D = self.m.B, self.m.S, self.m.D
+        self.h_hidden0 = pin(hidden0)
+        self.h_rows = [pin(r) for r in rows_np]
+        self.h_sets = [pin(torch.as_tensor(g, dtype=torch.int32)) for g in sets_np]
+        self.h_out_rows = [torch.empty(B, g.shape[1], D, dtype=torch.float32).pin_memory() for g in self.h_sets]
+        self.h_refresh = torch.empty(B * S, dtype=torch.int32).pin_memory()
+        self.max_new = max(g.shape[1] for g in self.h_sets)
+        self.staging = torch.empty(self.m.staging_bytes(self.max_new), dtype=torch.uint8, device="cuda")
+
+    def run_host(self, stream=None):
+        """The same generation through marche_step_host: every step copies its inputs from
+        pinned host memory and its results back.  Returns (h2d_bytes, d2h_bytes) per generation."""
+        m, B, D = self.m, self.m.B, self.m.D
+        self.hidden.copy_(self.h_hidden0, non_blocking=True)
+        h2d = self.h_hidden0.numel() * 4
+        d2h = 0
+        m.init_cache(self.cache, stream)
+        k_prev = 0
+        for t in range(self.T):
+            prev_rows = self.h_rows[t - 1] if t > 0 else None
+            prev_idx = self.h_sets[t - 1] if t > 0 else None
+            excl = self.h_sets[t + 1] if t + 1 < self.T else None
+            k = m.step_host(t == 0, self.hidden, self.cache, prev_rows, prev_idx, self.h_sets[t], excl,
+                            self.refresh_flat[(t - 1) % 2], k_prev, self.ratio, self.hidden_out,
+                            self.refresh_flat[t % 2], self.h_out_rows[t], self.h_refresh, self.max_new, self.staging,
+                            self.workspace, stream)
+            n_new = self.h_sets[t].shape[1]
+            n_prev = 0 if prev_idx is None else prev_idx.shape[1]
+            n_excl = 0 if excl is None else excl.shape[1]
+            h2d += B * n_prev * D * 4 + 4 * B * (n_prev + n_new + n_excl)
+            d2h += B * n_new * D * 4 + 4 * B * k
+            k_prev = k
+        return h2d, d2h

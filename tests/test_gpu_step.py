@@ -168,6 +168,35 @@ def test_full_ratio_equals_full_recompute():
     assert max_abs(host(cache_m), host(gen.cache)) <= 2e-2
 
 
+def test_host_driven_step_matches_device_loop():
+    """marche_step_host (inputs and results in host buffers) reproduces the device-resident
+    loop bit for bit: same kernels, same order; only the copies differ."""
+    cfg = synth.CONFIGS["tiny"].replace(dtype="bf16")
+    blocks = synth.make_weights(cfg)
+    hidden0 = synth.make_hidden(cfg)
+    sets = synth.new_token_sets(cfg, synth.generation_orders(cfg))
+    rows = [synth.replacement_rows(cfg, t, sets[t].shape[1]) for t in range(cfg.T)]
+    m, gen = gpu_generation(cfg, blocks, sets, 0.1)
+    log = gen.run(dev(hidden0), record=True)
+    gen.alloc_host_buffers(hidden0, rows, sets)
+    h2d, d2h = gen.run_host()
+    torch.cuda.synchronize()
+    assert h2d > hidden0.nbytes and d2h > 0
+    for t, rec in enumerate(log):
+        for b in range(cfg.B):
+            assert np.array_equal(gen.h_out_rows[t][b].numpy(), rec["hidden_out"][b, sets[t][b]])
+    k = log[-1]["refresh"].shape[1]
+    assert np.array_equal(gen.h_refresh[: cfg.B * k].view(cfg.B, k).numpy(), log[-1]["refresh"])
+    # profiling hooks: every launch is charged to a class, and the counter agrees
+    n0 = m.launch_count()
+    m.profile_begin()
+    gen.run(dev(hidden0))
+    prof = m.profile_end()
+    assert sum(v[1] for v in prof.values()) == m.launch_count() - n0
+    assert prof["attention"][1] == cfg.L * cfg.T and prof["gemm_qkv"][1] == cfg.L * cfg.T
+    assert all(v[0] >= 0 for v in prof.values())
+
+
 def test_argument_errors():
     cfg = synth.CONFIGS["tiny"]
     blocks = synth.make_weights(cfg)
