@@ -250,13 +250,14 @@ def run_ours(args, cfg):
             dist.all_reduce(ms, op=dist.ReduceOp.MAX)
         return float(ms.item()) / reps
 
+    n_dec = args.decode_steps or None
     for _ in range(args.warmup):
-        gen.run(hidden0)
+        gen.run(hidden0, n_steps=n_dec)
     torch.cuda.synchronize()
     clocks = ClockSampler(local)
     clocks.start()
     launches0 = m.launch_count()
-    ms_gen = timed(lambda: gen.run(hidden0), args.steps)
+    ms_gen = timed(lambda: gen.run(hidden0, n_steps=n_dec), args.steps)
     launches = m.launch_count() - launches0
     clock_info = clocks.stop()
     assert m.device_status() == 0, "a bounded device wait gave up"
@@ -339,6 +340,8 @@ def main():
     ap.add_argument("--blocks", type=int, default=0, help="override the depth (profiling captures only)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling captures only)")
     ap.add_argument("--tsteps", type=int, default=0, help="override the decoding steps (profiling captures only)")
+    ap.add_argument("--decode-steps", type=int, default=0,
+                    help="stop each generation after this many decoding steps (profiling captures only)")
     ap.add_argument("--no-extras", action="store_true", help="only the timed region (for ncu launch lists)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -36,7 +36,7 @@ class Generation:
         self.scores = torch.empty(B, S, dtype=torch.float32, device=dev)
 
     def run(self, hidden0: torch.Tensor, mode: str = "marche", record: bool = False,
-            forced_refresh: Optional[List[torch.Tensor]] = None, stream=None):
+            forced_refresh: Optional[List[torch.Tensor]] = None, stream=None, n_steps: Optional[int] = None):
         """Enqueues all T steps.  mode "full" runs the full-recompute baseline.  With
         record=True returns per-step host copies (this synchronises every step)."""
         m, B = self.m, self.m.B
@@ -44,7 +44,7 @@ class Generation:
         m.init_cache(self.cache, stream)
         log = []
         k_prev = 0
-        for t in range(self.T):
+        for t in range(self.T if n_steps is None else min(n_steps, self.T)):
             G = self.new_sets[t]
             X = self.new_sets[t + 1] if t + 1 < self.T else None
             R_out = self.refresh_flat[t % 2]
