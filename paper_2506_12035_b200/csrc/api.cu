@@ -33,6 +33,7 @@ struct marche_ctx {
   float eps = 1e-6f;
   int score_layer = 0;
   bool force_simt = false;
+  int gemm_mode = 0;                                  // 0 auto, 1 single-CTA MMA, 2 CTA-pair MMA (MARCHE_GEMM)
   std::vector<std::pair<const void*, bool>> caches;  // (cache pointer, filled)
   int* status_host = nullptr;                         // pinned, mapped
   int* status_dev = nullptr;
@@ -106,7 +107,10 @@ int do_linear(marche_ctx* ctx, int cls, const void* a, int lda, int M, const voi
   if (M > 0) mark(ctx, cls, st);
   const bool tc = ctx->bf16 && !ctx->force_simt && N % 128 == 0 && K % 64 == 0 && lda % 8 == 0 &&
                   (((uintptr_t)a | (uintptr_t)w | (uintptr_t)out) & 15) == 0;
-  if (tc)
+  const bool pair = tc && (ctx->gemm_mode == 2 || (ctx->gemm_mode == 0 && M > 128));
+  if (pair)
+    MARCHE_TRY(launch_gemm_tcgen05_2cta(a, lda, M, w, bias, N, K, epi, out, ctx->status_dev, st), "gemm_tcgen05_2cta");
+  else if (tc)
     MARCHE_TRY(launch_gemm_tcgen05(a, lda, M, w, bias, N, K, epi, out, ctx->status_dev, st), "gemm_tcgen05");
   else
     MARCHE_TRY(launch_gemm_simt(ctx->bf16, a, lda, M, w, bias, N, K, epi, out, st), "gemm");
@@ -228,6 +232,8 @@ int marche_create(const marche_config* cfg, const marche_block_weights* blocks, 
   ctx->score_layer = sl;
   const char* fs = getenv("MARCHE_FORCE_SIMT");
   ctx->force_simt = fs && fs[0] == '1';
+  const char* gm = getenv("MARCHE_GEMM");
+  ctx->gemm_mode = gm ? atoi(gm) : 0;
   cudaError_t e = cudaGetDevice(&ctx->device);
   if (e == cudaSuccess) e = cudaHostAlloc((void**)&ctx->status_host, 64, cudaHostAllocMapped);
   if (e == cudaSuccess) {

@@ -41,6 +41,24 @@ MARCHE_DEVINL float warp_max(float v) {
 // Exact (erf) GELU, the flavour the block uses.
 MARCHE_DEVINL float gelu_erf(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752440f)); }
 
+// GELU for the bf16 tensor-core epilogue: erf by the 5-term rational-exponential formula
+// erf(x) = 1 - (a1 t + ... + a5 t^5) exp(-x^2), t = 1/(1 + p x) (absolute error <= 1.5e-7, far
+// below the bf16 rounding of the result), about a third of the instructions of erff().
+MARCHE_DEVINL float gelu_erf_fast(float x) {
+  const float z = fabsf(x) * 0.70710678118654752440f;
+  float t;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f, z, 1.0f)));
+  float poly = fmaf(1.061405429f, t, -1.453152027f);
+  poly = fmaf(poly, t, 1.421413741f);
+  poly = fmaf(poly, t, -0.284496736f);
+  poly = fmaf(poly, t, 0.254829592f);
+  float ex;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(ex) : "f"(-z * z * 1.4426950408889634f));
+  const float e = poly * t * ex;                      // 1 - erf(z), z >= 0
+  const float cdf = x >= 0.f ? 1.0f - 0.5f * e : 0.5f * e;
+  return x * cdf;
+}
+
 // Stores 4 consecutive outputs of type T starting at a 4-element aligned column.
 MARCHE_DEVINL void store4(float* p, float a, float b, float c, float d) {
   *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);

@@ -9,13 +9,15 @@
 //                        in TMEM), frees ring slots and publishes accumulators with
 //                        tcgen05.commit
 //   warps 2-5            epilogue: tcgen05.ld of the accumulator (thread = output row),
-//                        bias / GELU / fp32 residual, stores
+//                        bias / GELU, swizzled staging box in shared memory, TMA bulk store
+//                        (TMA reduce-add for the fp32 residual)
 // The accumulator is double-buffered in TMEM (2 x BN columns) so the epilogue of tile i
 // overlaps the MMAs of tile i+1.  Rows beyond M are zero-filled by TMA on load and
 // masked on store, so M needs no padding.  Every mbarrier wait is bounded; on a
 // give-up the kernel records a status code and drains instead of hanging.
 #include <cuda.h>
 
+#include "gemm_epilogue.cuh"
 #include "kernels.h"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"
@@ -33,7 +35,8 @@ template <int BN> struct GemmCfg {
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGES = (BN == 256) ? 4 : 6;
   static constexpr int RING_BYTES = STAGES * (A_BYTES + B_BYTES);
-  static constexpr int SMEM_BYTES = RING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int STAGING_BYTES = 4 * 4096;            // one 32-row x 128-byte box per epilogue warp
+  static constexpr int SMEM_BYTES = RING_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
   static constexpr int TMEM_COLS = 2 * BN;
 };
 
@@ -42,8 +45,8 @@ enum { ST_PRODUCER = 0x11, ST_MMA = 0x12, ST_EPILOGUE = 0x13 };
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
-                    int M, int N, int K, const float* __restrict__ bias, void* __restrict__ out_,
-                    int* __restrict__ status) {
+                    const __grid_constant__ CUtensorMap tmap_out, int M, int N, int K,
+                    const float* __restrict__ bias, int* __restrict__ status) {
   using Cfg = GemmCfg<BN>;
   constexpr int STAGES = Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
@@ -51,14 +54,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   const uint32_t base = (raw + 1023u) & ~1023u;             // swizzled tiles need 1024-byte alignment
   const uint32_t a_base = base;
   const uint32_t w_base = base + STAGES * A_BYTES;
-  const uint32_t bar_base = base + Cfg::RING_BYTES;         // 8-byte barriers
+  const uint32_t staging = base + Cfg::RING_BYTES;
+  const uint32_t bar_base = staging + Cfg::STAGING_BYTES;   // 8-byte barriers
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
   uint8_t* gen_base = smem_raw + (base - raw);
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + Cfg::RING_BYTES + 8 * (2 * STAGES + 4));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + Cfg::RING_BYTES + 8 * (2 * STAGES + 4) + 8);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + Cfg::RING_BYTES + Cfg::STAGING_BYTES + 8 * (2 * STAGES + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + Cfg::RING_BYTES + Cfg::STAGING_BYTES + 8 * (2 * STAGES + 4) + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_m = (M + BM - 1) / BM, n_n = N / BN, n_tiles = n_m * n_n, n_kb = K / BK;
@@ -91,6 +95,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     if (lane == 0) {
       ptx::prefetch_tensormap(&tmap_a);
       ptx::prefetch_tensormap(&tmap_w);
+      ptx::prefetch_tensormap(&tmap_out);
       int it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -153,54 +158,22 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       const uint32_t acc_ph = (uint32_t)(tile_i >> 1) & 1u;
       if (!ptx::mbar_wait(tfull_bar(acc), acc_ph, abort_flag)) { ok = false; break; }
       ptx::tc_fence_after();
-      const int row = m_blk * BM + quarter * 32 + lane;
+      const int row0 = m_blk * BM + quarter * 32;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+      const uint32_t my_stage = staging + (uint32_t)(warp - 2) * 4096u;
+      if (row0 < M) {
+        constexpr int EC = EpiCols<EPI>::value;
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t r[32];
-        ptx::tmem_ld_32x32(t_row + (uint32_t)(c * 32), r);
-        ptx::tmem_ld_wait();
-        const int col = n_blk * BN + c * 32;
-        if (row < M) {
-          const float4* b4 = reinterpret_cast<const float4*>(bias + col);
-          if (EPI == 1) {
-            float4* o4 = reinterpret_cast<float4*>(reinterpret_cast<float*>(out_) + (size_t)row * N + col);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const float4 bv = __ldg(b4 + j);
-              float4 o = o4[j];
-              o.x += __uint_as_float(r[4 * j + 0]) + bv.x;
-              o.y += __uint_as_float(r[4 * j + 1]) + bv.y;
-              o.z += __uint_as_float(r[4 * j + 2]) + bv.z;
-              o.w += __uint_as_float(r[4 * j + 3]) + bv.w;
-              o4[j] = o;
-            }
-          } else {
-            uint4* o4 = reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(out_) + (size_t)row * N + col);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const float4 b0 = __ldg(b4 + 2 * j), b1 = __ldg(b4 + 2 * j + 1);
-              float v0 = __uint_as_float(r[8 * j + 0]) + b0.x, v1 = __uint_as_float(r[8 * j + 1]) + b0.y;
-              float v2 = __uint_as_float(r[8 * j + 2]) + b0.z, v3 = __uint_as_float(r[8 * j + 3]) + b0.w;
-              float v4 = __uint_as_float(r[8 * j + 4]) + b1.x, v5 = __uint_as_float(r[8 * j + 5]) + b1.y;
-              float v6 = __uint_as_float(r[8 * j + 6]) + b1.z, v7 = __uint_as_float(r[8 * j + 7]) + b1.w;
-              if (EPI == 2) {
-                v0 = gelu_erf(v0); v1 = gelu_erf(v1); v2 = gelu_erf(v2); v3 = gelu_erf(v3);
-                v4 = gelu_erf(v4); v5 = gelu_erf(v5); v6 = gelu_erf(v6); v7 = gelu_erf(v7);
-              }
-              uint4 pk;
-              pk.x = pack_bf16x2(v0, v1); pk.y = pack_bf16x2(v2, v3);
-              pk.z = pack_bf16x2(v4, v5); pk.w = pack_bf16x2(v6, v7);
-              o4[j] = pk;
-            }
-          }
-        }
+        for (int c0 = 0; c0 < BN; c0 += EC)
+          epilogue_box<EPI>(t_row + (uint32_t)c0, bias + n_blk * BN + c0, &tmap_out, n_blk * BN + c0, row0, my_stage,
+                            lane);
       }
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
     }
     if (!ok && lane == 0) *(volatile int*)status = ST_EPILOGUE;
+    if (lane == 0) ptx::bulk_wait_all();                    // this warp's stores have landed
   }
 
   ptx::tc_fence_before();
@@ -223,8 +196,8 @@ bool make_map_2d(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols
 int sm_count() { return device_sm_count(); }
 
 template <int BN, int EPI>
-cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tw, int M, int N, int K, const float* bias,
-                       void* out, int* status, cudaStream_t st) {
+cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& to, int M, int N, int K,
+                       const float* bias, int* status, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -234,7 +207,7 @@ cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tw, int M, int 
   }
   const int n_tiles = ((M + BM - 1) / BM) * (N / BN);
   const int grid = n_tiles < sm_count() ? n_tiles : sm_count();
-  gemm_tcgen05_kernel<BN, EPI><<<grid, kGemmThreads, GemmCfg<BN>::SMEM_BYTES, st>>>(ta, tw, M, N, K, bias, out, status);
+  gemm_tcgen05_kernel<BN, EPI><<<grid, kGemmThreads, GemmCfg<BN>::SMEM_BYTES, st>>>(ta, tw, to, M, N, K, bias, status);
   return cudaGetLastError();
 }
 
@@ -254,11 +227,13 @@ cudaError_t launch_gemm_tcgen05(const void* a, int lda, int M, const void* w, co
   if (M == 0) return cudaSuccess;
   if (N % 128 || K % BK || lda % 8 || ((uintptr_t)a & 15) || ((uintptr_t)w & 15)) return cudaErrorInvalidValue;
   const int bn = gemm_tcgen05_pick_bn(M, N);
-  CUtensorMap ta, tw;
+  CUtensorMap ta, tw, to;
   if (!make_map_2d(&ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM)) return cudaErrorInvalidValue;
   if (!make_map_2d(&tw, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)bn)) return cudaErrorInvalidValue;
+  if (((uintptr_t)out & 15) || !tma_make_store_map(&to, out, (uint64_t)M, (uint64_t)N, epilogue == 1 ? 4 : 2))
+    return cudaErrorInvalidValue;
 #define MARCHE_GEMM_CASE(BN_, EPI_) \
-  if (bn == BN_ && epilogue == EPI_) return launch_one<BN_, EPI_>(ta, tw, M, N, K, bias, out, status, st);
+  if (bn == BN_ && epilogue == EPI_) return launch_one<BN_, EPI_>(ta, tw, to, M, N, K, bias, status, st);
   MARCHE_GEMM_CASE(256, 0) MARCHE_GEMM_CASE(256, 1) MARCHE_GEMM_CASE(256, 2)
   MARCHE_GEMM_CASE(128, 0) MARCHE_GEMM_CASE(128, 1) MARCHE_GEMM_CASE(128, 2)
 #undef MARCHE_GEMM_CASE

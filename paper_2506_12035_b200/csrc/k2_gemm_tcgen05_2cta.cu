@@ -1,0 +1,252 @@
+// K2, 2-CTA flavour: the same projections as k2_gemm_tcgen05.cu with tcgen05.mma
+// cta_group::2.  Two CTAs on neighbouring SMs (a cluster of 2) share one 256 x BN output
+// tile: each CTA loads its own 128 rows of A and HALF of the W tile per K step, the pair's
+// tensor cores read both halves, and each CTA keeps its 128 x BN accumulator in its own
+// TMEM.  Per CTA a ring stage is 32 KB instead of 48 KB for the same MMA work, so the ring
+// hides more TMA latency per byte of shared memory and L2 -> shared-memory traffic per flop
+// drops by a third.  No TMA multicast is used: every CTA fetches its own tiles.
+//
+// Protocol (rank 0 of the pair is the leader, rank 1 the peer):
+//   full[s]    leader's barrier; the leader's producer arms it with the bytes of BOTH CTAs'
+//              tiles and both producers' TMA loads complete on it
+//   empty[s]   one per CTA; the leader's MMA thread frees a slot in both CTAs with one
+//              multicast tcgen05.commit
+//   tfull[a]   one per CTA; multicast commit when an accumulator is complete
+//   tempty[a]  leader's barrier; the 8 epilogue warps of each CTA arrive (remotely for the peer)
+// Epilogue: TMEM -> registers -> swizzled staging box in shared memory -> TMA bulk store (TMA
+// reduce-add for the fp32 residual), see gemm_epilogue.cuh.
+// All waits are bounded; both CTAs meet at a final cluster barrier so that neither exits
+// while its shared memory or TMEM can still be touched by the other.
+#include <cuda.h>
+
+#include <cstdlib>
+
+#include "gemm_epilogue.cuh"
+#include "kernels.h"
+#include "sm100_ptx.cuh"
+#include "tma_host.h"
+
+namespace marche {
+
+namespace {
+
+constexpr int BM = 128;                   // rows per CTA (256 per pair)
+constexpr int BK = 64;
+constexpr int kThreads = 320;             // producer warp, MMA warp, 8 epilogue warps
+constexpr int A_BYTES = BM * BK * 2;
+
+template <int BN> struct PairCfg {
+  static constexpr int BH_BYTES = (BN / 2) * BK * 2;            // this CTA's half of the W tile
+  static constexpr int STAGE_BYTES = A_BYTES + BH_BYTES;
+  static constexpr int STAGES = (BN == 256) ? 5 : 6;
+  static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
+  static constexpr int STAGING_BYTES = 8 * 4096;                 // one 32-row x 128-byte box per epilogue warp
+  static constexpr int SMEM_BYTES = RING_BYTES + STAGING_BYTES + 1024 + 256;
+  static constexpr int TMEM_COLS = 2 * BN;
+};
+
+enum { ST2_PRODUCER = 0x31, ST2_MMA = 0x32, ST2_EPILOGUE = 0x33 };
+
+template <int BN, int EPI>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
+                         const __grid_constant__ CUtensorMap tmap_out, int M, int N, int K,
+                         const float* __restrict__ bias, int* __restrict__ status) {
+  using Cfg = PairCfg<BN>;
+  constexpr int STAGES = Cfg::STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = ptx::smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  const uint32_t staging = base + Cfg::RING_BYTES;
+  const uint32_t bar_base = staging + Cfg::STAGING_BYTES;
+  auto a_tile = [&](int s) { return base + (uint32_t)s * Cfg::STAGE_BYTES; };
+  auto w_tile = [&](int s) { return base + (uint32_t)s * Cfg::STAGE_BYTES + A_BYTES; };
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+  uint8_t* gen_base = smem_raw + (base - raw);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + Cfg::RING_BYTES + Cfg::STAGING_BYTES + 8 * (2 * STAGES + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + Cfg::RING_BYTES + Cfg::STAGING_BYTES + 8 * (2 * STAGES + 4) + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = ptx::cluster_ctarank();           // 0 = leader
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int n_m2 = (M + 2 * BM - 1) / (2 * BM), n_n = N / BN, n_tiles = n_m2 * n_n, n_kb = K / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(full_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(tfull_bar(a), 1);
+      ptx::mbar_init(tempty_bar(a), 16);                  // 8 epilogue warps x 2 CTAs
+    }
+    abort_flag[0] = 0;
+    abort_flag[1] = 0;
+    ptx::fence_barrier_init();
+    ptx::fence_proxy_async();
+  }
+  if (warp == 2) {
+    ptx::tmem_alloc_pair(ptx::smem_u32((const void*)tmem_slot), Cfg::TMEM_COLS);
+    ptx::tmem_relinquish_pair();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync_all();                                // both CTAs' barriers exist before any remote signal
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer (both CTAs)
+    if (lane == 0) {
+      ptx::prefetch_tensormap(&tmap_a);
+      ptx::prefetch_tensormap(&tmap_w);
+      ptx::prefetch_tensormap(&tmap_out);
+      int it = 0;
+      bool ok = true;
+      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+        const int m2 = tile / n_n, n_blk = tile - m2 * n_n;
+        const int row0 = m2 * 2 * BM + (int)rank * BM;                // this CTA's 128 rows of A
+        const int wrow0 = n_blk * BN + (int)rank * (BN / 2);          // this CTA's half of the W tile
+        for (int kb = 0; kb < n_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+          if (!ptx::mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t leader_full = ptx::mapa(full_bar(s), 0);
+          if (rank == 0) ptx::mbar_expect_tx(full_bar(s), 2 * Cfg::STAGE_BYTES);
+          ptx::tma_load_2d_pair(a_tile(s), &tmap_a, kb * BK, row0, leader_full);
+          ptx::tma_load_2d_pair(w_tile(s), &tmap_w, kb * BK, wrow0, leader_full);
+        }
+      }
+      if (!ok) *(volatile int*)status = ST2_PRODUCER;
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer (leader only)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = ptx::idesc_bf16_f32(2 * BM, BN);
+      int it = 0, tile_i = 0;
+      bool ok = true;
+      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++tile_i) {
+        const int acc = tile_i & 1;
+        const uint32_t acc_ph = (uint32_t)(tile_i >> 1) & 1u;
+        if (!ptx::mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < n_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+          if (!ptx::mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+          ptx::tc_fence_after();
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t da = ptx::smem_desc_k_sw128(a_tile(s) + k * 32);
+            const uint64_t dw = ptx::smem_desc_k_sw128(w_tile(s) + k * 32);
+            ptx::umma_f16_pair(d_tmem, da, dw, idesc, (kb | k) ? 1u : 0u);
+          }
+          ptx::umma_commit_pair(empty_bar(s), 3);           // frees the slot in both CTAs
+        }
+        if (ok) ptx::umma_commit_pair(tfull_bar(acc), 3);   // accumulator complete in both CTAs
+      }
+      if (!ok) *(volatile int*)status = ST2_MMA;
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue (warps 2..9, both CTAs)
+    const int quarter = warp & 3;                           // TMEM lanes 32*quarter .. +31
+    const int half = (warp - 2) >> 2;                       // which half of the BN columns
+    int tile_i = 0;
+    bool ok = true;
+    for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++tile_i) {
+      const int m2 = tile / n_n, n_blk = tile - m2 * n_n;
+      const int acc = tile_i & 1;
+      const uint32_t acc_ph = (uint32_t)(tile_i >> 1) & 1u;
+      if (!ptx::mbar_wait(tfull_bar(acc), acc_ph, abort_flag)) { ok = false; break; }
+      ptx::tc_fence_after();
+      const int row0 = m2 * 2 * BM + (int)rank * BM + quarter * 32;
+      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+      const uint32_t my_stage = staging + (uint32_t)(warp - 2) * 4096u;
+      if (row0 < M) {
+        constexpr int EC = EpiCols<EPI>::value;
+#pragma unroll 1
+        for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += EC)
+          epilogue_box<EPI>(t_row + (uint32_t)c0, bias + n_blk * BN + c0, &tmap_out, n_blk * BN + c0, row0, my_stage,
+                            lane);
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa(tempty_bar(acc), 0));
+    }
+    if (!ok && lane == 0) *(volatile int*)status = ST2_EPILOGUE;
+    if (lane == 0) ptx::bulk_wait_all();                    // this warp's stores have left shared memory and landed
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync_all();                                  // peer done with our smem / TMEM and vice versa
+  if (warp == 2) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc_pair(tmem_base, Cfg::TMEM_COLS);
+  }
+}
+
+bool make_map_2d(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
+  const uint64_t dims[2] = {cols, rows};
+  const uint64_t strides[1] = {ld * 2};
+  const uint32_t box[2] = {BK, box_rows};
+  return tma_make_map_bf16(map, ptr, 2, dims, strides, box, true);
+}
+
+template <int BN, int EPI>
+cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& to, int M, int N, int K,
+                        const float* bias, int* status, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_2cta_kernel<BN, EPI>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<BN>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int n_tiles = ((M + 2 * BM - 1) / (2 * BM)) * (N / BN);
+  const int max_pairs = device_sm_count() / 2;
+  const int pairs = n_tiles < max_pairs ? n_tiles : max_pairs;
+  gemm_tcgen05_2cta_kernel<BN, EPI><<<2 * pairs, kThreads, PairCfg<BN>::SMEM_BYTES, st>>>(ta, tw, to, M, N, K, bias,
+                                                                                         status);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+// Tile width: 256 whenever N allows it.  Measured on B200 at M = 4.3-5.8 k rows, the 128-wide
+// pair tile costs about 0.7x a 256-wide one (1.5x the operand bytes per flop), so it never wins
+// back what it gains in wave balance.  MARCHE_BN=128 overrides (measurement only).
+int gemm_tcgen05_2cta_pick_bn(int M, int N) {
+  static int forced = -1;
+  if (forced < 0) {
+    const char* e = getenv("MARCHE_BN");
+    forced = e ? atoi(e) : 0;
+  }
+  (void)M;
+  if (N % 256) return 128;
+  return forced == 128 ? 128 : 256;
+}
+
+cudaError_t launch_gemm_tcgen05_2cta(const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
+                                     int epilogue, void* out, int* status, cudaStream_t st) {
+  if (M == 0) return cudaSuccess;
+  if (N % 128 || K % BK || lda % 8 || ((uintptr_t)a & 15) || ((uintptr_t)w & 15)) return cudaErrorInvalidValue;
+  const int bn = gemm_tcgen05_2cta_pick_bn(M, N);
+  CUtensorMap ta, tw, to;
+  if (!make_map_2d(&ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM)) return cudaErrorInvalidValue;
+  if (!make_map_2d(&tw, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)(bn / 2))) return cudaErrorInvalidValue;
+  if (((uintptr_t)out & 15) || !tma_make_store_map(&to, out, (uint64_t)M, (uint64_t)N, epilogue == 1 ? 4 : 2))
+    return cudaErrorInvalidValue;
+#define MARCHE_GEMM2_CASE(BN_, EPI_) \
+  if (bn == BN_ && epilogue == EPI_) return launch_pair<BN_, EPI_>(ta, tw, to, M, N, K, bias, status, st);
+  MARCHE_GEMM2_CASE(256, 0) MARCHE_GEMM2_CASE(256, 1) MARCHE_GEMM2_CASE(256, 2)
+  MARCHE_GEMM2_CASE(128, 0) MARCHE_GEMM2_CASE(128, 1) MARCHE_GEMM2_CASE(128, 2)
+#undef MARCHE_GEMM2_CASE
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace marche

@@ -51,6 +51,10 @@ cudaError_t launch_gemm_simt(bool bf16_t, const void* a, int lda, int M, const v
 cudaError_t launch_gemm_tcgen05(const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
                                 int epilogue, void* out, int* status, cudaStream_t st);
 int gemm_tcgen05_pick_bn(int M, int N);
+// Same contract, tcgen05.mma cta_group::2: CTA pairs share 256 x BN tiles (cluster of 2, no multicast).
+cudaError_t launch_gemm_tcgen05_2cta(const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
+                                     int epilogue, void* out, int* status, cudaStream_t st);
+int gemm_tcgen05_2cta_pick_bn(int M, int N);
 
 // K3 (SIMT): attention of n queries per sample over all S cache rows.
 cudaError_t launch_attention_simt(bool bf16_t, const void* q, int ld_q, int B, int n, int S, int H, int dh,

@@ -46,6 +46,20 @@ inline bool tma_make_map_bf16(CUtensorMap* map, const void* ptr, int rank, const
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Row-major [rows][cols] matrix of bf16 (elem_bytes 2) or fp32 (4) as the target of 32-row boxes
+// that are 128 bytes wide (64 bf16 or 32 fp32 columns), 128-byte swizzle.
+inline bool tma_make_store_map(CUtensorMap* map, void* ptr, uint64_t rows, uint64_t cols, int elem_bytes) {
+  EncodeTiledFn fn = tma_encode_fn();
+  if (!fn) return false;
+  const cuuint64_t d[2] = {cols, rows};
+  const cuuint64_t s[1] = {cols * (uint64_t)elem_bytes};
+  const cuuint32_t b[2] = {(cuuint32_t)(128 / elem_bytes), 32};
+  const cuuint32_t e[2] = {1, 1};
+  return fn(map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, ptr, d, s, b,
+            e, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 inline int device_sm_count() {
   static int n = 0;
   if (!n) {
