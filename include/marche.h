@@ -180,6 +180,29 @@ int marche_select_refresh(marche_ctx* ctx, const float* scores,
                           const int32_t* exclude_idx, int n_excl,
                           int k, int32_t* refresh_idx, void* mask_scratch, marche_stream stream);
 
+/* The same selection as marche_select_refresh for callers that have no scratch buffer to give
+ * and cannot obtain one: code running where device allocation is not allowed (inside a region
+ * whose memory was sized up front, a latency-critical serving loop that must never touch the
+ * allocator, a plug-in that is handed only its input and output tensors).  The paper has no
+ * counterpart; this is a packaging variant of the same kernels.
+ *   - The candidate mask lives in a fixed array inside the library, MARCHE_STATIC_SCRATCH_BYTES
+ *     (256 KiB) per GPU, which every GPU that loads the library holds until the process exits.
+ *     batch*seq_len must not exceed that size; otherwise MARCHE_EWORKSPACE is returned, nothing
+ *     is enqueued and marche_last_error() names both numbers.
+ *   - No device memory is allocated or freed by this call, now or later.  Its first call on a
+ *     device looks up the array's device address (a synchronous, one-time driver query), so make
+ *     that first call before starting any stream capture on that device.
+ *   - All calls on a device, from every context, share the one array and it keeps the bytes of
+ *     the last call.  Each call rewrites every byte it reads, so stale contents are harmless, but
+ *     two calls whose kernels overlap on the GPU (different streams, no dependency) race on it:
+ *     keep them on one stream or order them with events.
+ * Arguments, result and errors otherwise exactly as marche_select_refresh without mask_scratch. */
+#define MARCHE_STATIC_SCRATCH_BYTES (256 * 1024)
+int marche_select_refresh_static(marche_ctx* ctx, const float* scores,
+                                 const int32_t* new_idx, int n_new,
+                                 const int32_t* exclude_idx, int n_excl,
+                                 int k, int32_t* refresh_idx, marche_stream stream);
+
 /* Copies the relevance scores float [B][S] that the last step left in
  * `workspace` to `scores_out` (device).  Section 4.2: attention probability
  * from the generating tokens to each token, summed over heads and queries. */

@@ -50,6 +50,7 @@ _SIGNATURES = {
     "marche_step": (C.c_int, [_vp, _vp, _vp, _vp, _i, _vp, _i, _vp, _i, _f, _vp, _vp, C.POINTER(C.c_int), _vp, _sz, _vp]),
     "marche_full_step": (C.c_int, [_vp, _vp, _vp, _vp, _i, _vp, _i, _f, _vp, _vp, C.POINTER(C.c_int), _vp, _sz, _vp]),
     "marche_select_refresh": (C.c_int, [_vp, _vp, _vp, _i, _vp, _i, _i, _vp, _vp, _vp]),
+    "marche_select_refresh_static": (C.c_int, [_vp, _vp, _vp, _i, _vp, _i, _i, _vp, _vp]),
     "marche_get_scores": (C.c_int, [_vp, _vp, _vp, _vp]),
     "marche_build_active": (C.c_int, [_vp, _vp, _i, _vp, _i, _vp, _i, _vp, _vp]),
     "marche_scatter_rows": (C.c_int, [_vp, _vp, _vp, _i, _vp, _vp]),
@@ -209,6 +210,17 @@ class Marche:
             self.h, _ptr(scores), _ptr(new_idx), 0 if new_idx is None else new_idx.shape[1],
             _ptr(exclude_idx), 0 if exclude_idx is None else exclude_idx.shape[1], k, _ptr(refresh_idx),
             _ptr(mask_scratch), _stream(stream)))
+
+    def select_refresh_static(self, scores, new_idx, exclude_idx, k, refresh_idx, stream=None):
+        """select_refresh without a caller-supplied scratch buffer: the candidate mask lives in a
+        fixed 256 KiB array inside the library (B*S must fit).  Nothing is allocated."""
+        rc = self.lib.marche_select_refresh_static(
+            self.h, _ptr(scores), _ptr(new_idx), 0 if new_idx is None else new_idx.shape[1],
+            _ptr(exclude_idx), 0 if exclude_idx is None else exclude_idx.shape[1], k, _ptr(refresh_idx),
+            _stream(stream))
+        if rc == -3:
+            raise MarcheError(rc, self.lib.marche_last_error(self.h).decode())
+        self._check(rc)
 
     def get_scores(self, workspace, scores_out, stream=None):
         self._check(self.lib.marche_get_scores(self.h, _ptr(workspace), _ptr(scores_out), _stream(stream)))

@@ -512,6 +512,62 @@ const char* marche_kernel_class_name(int cls) {
   return (cls >= 0 && cls < MARCHE_N_KERNEL_CLASSES) ? names[cls] : "?";
 }
 
+// ---------------------------------------------------------------- allocation-free selection
+// Candidate-mask scratch of marche_select_refresh_static.  It lives in the library image, so every
+// GPU that loads the library holds these bytes until the process exits.  In host code the name
+// below is only a stand-in for the device object; its device address is obtained once per device
+// with cudaGetSymbolAddress and handed to the kernels.
+static __device__ __align__(256) uint8_t g_static_mask_scratch[MARCHE_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+uint8_t* g_static_mask_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on the current device (looked up on first use).
+cudaError_t static_mask_address(uint8_t** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!g_static_mask_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_mask_scratch);
+    if (e != cudaSuccess) return e;
+    g_static_mask_ptr[dev] = static_cast<uint8_t*>(p);
+  }
+  *out = g_static_mask_ptr[dev];
+  return cudaSuccess;
+}
+}  // namespace
+
+int marche_select_refresh_static(marche_ctx* ctx, const float* scores, const int32_t* new_idx, int n_new,
+                                 const int32_t* exclude_idx, int n_excl, int k, int32_t* refresh_idx,
+                                 marche_stream stream) {
+  if (!ctx || !scores || n_new < 0 || n_excl < 0 || k < 0) return MARCHE_EINVAL;
+  if ((n_new > 0 && !new_idx) || (n_excl > 0 && !exclude_idx)) return MARCHE_EINVAL;
+  const int B = ctx->cfg.batch, S = ctx->cfg.seq_len;
+  if (k > S - n_new - n_excl) return MARCHE_EINVAL;
+  if ((size_t)B * (size_t)S > (size_t)MARCHE_STATIC_SCRATCH_BYTES) {
+    char msg[160];
+    snprintf(msg, sizeof msg, "marche_select_refresh_static: batch*seq_len = %zu exceeds the built-in scratch of %d bytes",
+             (size_t)B * (size_t)S, (int)MARCHE_STATIC_SCRATCH_BYTES);
+    ctx->last_error = msg;
+    return MARCHE_EWORKSPACE;
+  }
+  if (k == 0) return MARCHE_OK;
+  if (!refresh_idx) return MARCHE_EINVAL;
+  uint8_t* mask = nullptr;
+  MARCHE_TRY(static_mask_address(&mask), "cudaGetSymbolAddress");
+  cudaStream_t st = (cudaStream_t)stream;
+  // The mask kernel writes all B*S bytes it uses, so nothing left over from an earlier call
+  // (of this or any other context) can leak into this one.
+  mark(ctx, MARCHE_KC_FLAGS, st);
+  MARCHE_TRY(launch_step_flags(nullptr, 0, new_idx, n_new, exclude_idx, n_excl, B, S, nullptr, mask, st), "flags");
+  mark(ctx, MARCHE_KC_TOPK, st);
+  MARCHE_TRY(launch_topk(nullptr, 0, const_cast<float*>(scores), mask, B, S, k, refresh_idx, st), "topk");
+  return MARCHE_OK;
+}
+
 const char* marche_strerror(int code) {
   switch (code) {
     case MARCHE_OK: return "ok";
