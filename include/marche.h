@@ -17,14 +17,25 @@
  *            returns without waiting for it (asynchronous), except where noted.
  * Notation   B batch rows, S tokens per sample, D width = H heads x dh,
  *            F MLP width, L blocks, nA active tokens per sample, nG generating
- *            ("new") tokens per sample, M = B*nA rows.  `T` is the compute
- *            type selected by marche_config.dtype (float or bf16).
+ *            ("new") tokens per sample, M = B*nA rows.
+ * Types      marche_config.dtype selects two element types.  `T` (q/k/v and the
+ *            K/V cache, i.e. everything attention reads) is float or bf16.  `A`
+ *            (both operands of the four projections: the weight matrices, and the
+ *            activation matrices that feed them - LayerNorm output, attention
+ *            output, GELU output) is float, or IEEE fp16 in MARCHE_BF16 contexts:
+ *            with 16-bit operands the rounding of exactly these activations
+ *            dominates the end-to-end error (bf16 there gives max-abs 5e-2 at 32
+ *            blocks, above the 3e-2 bound; fp16 gives 7e-3), fp16 runs at the same
+ *            tensor-core rate and size, and the tensor core wants both operands
+ *            of one MMA in the same format.  |values| of A must stay below 65504
+ *            (N(0, 0.02) weights, LayerNorm outputs, convex combinations of V rows
+ *            and GELU outputs of normalised inputs do).
  * Index sets int32, device, row-major [B][n] with the same n for every sample;
  *            entries are token positions in [0, S), unique within a sample.
  * Layouts    hidden / hidden_out  float [B][S][D]
  *            K/V cache            T [L][2][B][S][D]; [l][0] holds K, [l][1] V;
  *                                 head h occupies columns h*dh .. (h+1)*dh-1
- *            weight matrices      T [out][in] row-major; LayerNorm parameters
+ *            weight matrices      A [out][in] row-major; LayerNorm parameters
  *                                 and all biases are float
  * Errors     0 (MARCHE_OK) on success, a negative MARCHE_E* code otherwise; no
  *            C++ exception crosses the boundary and no device code traps.  When
@@ -65,7 +76,7 @@ enum {
 enum {
   MARCHE_EPI_BIAS = 0,          /* out T[M][N]      = acc + bias                          */
   MARCHE_EPI_BIAS_RESIDUAL = 1, /* out float[M][N] += acc + bias   (read-modify-write)    */
-  MARCHE_EPI_BIAS_GELU = 2      /* out T[M][N]      = GELU_erf(acc + bias)                */
+  MARCHE_EPI_BIAS_GELU = 2      /* out A[M][N]      = GELU_erf(acc + bias)                */
 };
 
 /* Kernel classes of marche_profile_end / marche_kernel_class_name. */
@@ -272,14 +283,14 @@ int marche_validate_indices(marche_ctx* ctx, const int32_t* active_idx, int n_ac
 /* Gather + LayerNorm (Algorithm 1 line 5, input side): for r = b*n + j,
  *   x = src[b][idx ? idx[b][j] : j][:]   (src float [B][src_rows][D])
  *   x_out[r][:] = x                      (float [B*n][D], skipped when NULL)
- *   u_out[r][:] = (x-mean)/sqrt(var+eps)*gamma + beta   (T [B*n][D])
+ *   u_out[r][:] = (x-mean)/sqrt(var+eps)*gamma + beta   (A [B*n][D])
  * Statistics in fp32 from the row held in registers (two passes). */
 int marche_gather_layernorm(marche_ctx* ctx, const float* src, int src_rows, const int32_t* idx, int n,
                             const float* gamma, const float* beta, float* x_out, void* u_out,
                             marche_stream stream);
 
-/* out = epilogue(a * w^T + bias): a T [M][K] with row stride lda elements,
- * w T [N][K], bias float [N], out [M][N] dense (type per epilogue).  The QKV,
+/* out = epilogue(a * w^T + bias): a A [M][K] with row stride lda elements,
+ * w A [N][K], bias float [N], out [M][N] dense (type per epilogue).  The QKV,
  * output and MLP projections on active rows only (Algorithm 1 lines 5 and 9).
  * bf16: K % 64 == 0, N % 128 == 0, lda % 8 == 0.  fp32 accumulation. */
 int marche_linear(marche_ctx* ctx, const void* a, int lda, int M, const void* w, const float* bias,
@@ -296,7 +307,7 @@ int marche_scatter_kv(marche_ctx* ctx, const void* k, const void* v, int ld_kv,
  * (Algorithm 1 lines 6-8, equal to Eq. 5 by Appendix A once the fresh K, V of
  * the active rows are in the cache), with the fused relevance reduction of
  * Section 4.2:
- *   q T [B*n][D] with row stride ld_q; o T [B*n][D] dense;
+ *   q T [B*n][D] with row stride ld_q; o A [B*n][D] dense;
  *   is_new  device uint8 [B][n] flags of the scoring queries, or NULL: no scores;
  *   score_partial device float [B][H][S]: per head, sum over flagged queries of
  *   the softmax weights (overwritten, not accumulated); ignored when is_new NULL. */

@@ -106,8 +106,9 @@ def _stream(stream: Optional[torch.cuda.Stream]) -> Optional[int]:
 
 def upload_weights(blocks: Sequence[Dict], dtype: str, device="cuda") -> List[Dict[str, torch.Tensor]]:
     """Copies per-block parameter arrays (NumPy or torch, fp32) to the device: the four
-    matrices in the compute type, LayerNorm parameters and biases in fp32."""
-    mt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    matrices as projection operands (fp16 in 16-bit mode, else fp32), LayerNorm parameters and
+    biases in fp32."""
+    mt = torch.float16 if dtype == "bf16" else torch.float32
     out = []
     for blk in blocks:
         d = {}
@@ -130,7 +131,8 @@ class Marche:
         self.lib = load_library()
         self.L, self.E, self.D, self.H, self.F, self.S, self.B = L, E, D, H, F, S, B
         self.dtype = dtype
-        self.torch_dtype = torch.bfloat16 if dtype == "bf16" else torch.float32
+        self.torch_dtype = torch.bfloat16 if dtype == "bf16" else torch.float32      # q/k/v, K/V cache
+        self.operand_dtype = torch.float16 if dtype == "bf16" else torch.float32     # projection operands
         self.weights = list(weights)          # keeps the device tensors alive
         assert len(self.weights) == L
         cfg = MarcheConfig(L, E, D, H, D // H, F, S, n_buffer, B, MARCHE_BF16 if dtype == "bf16" else MARCHE_F32,
@@ -139,7 +141,7 @@ class Marche:
         for l, blk in enumerate(self.weights):
             for name in BLOCK_FIELDS:
                 t = blk[name]
-                want = self.torch_dtype if name in MATRIX_FIELDS else torch.float32
+                want = self.operand_dtype if name in MATRIX_FIELDS else torch.float32
                 assert t.is_cuda and t.is_contiguous() and t.dtype == want, name
                 setattr(arr[l], name, t.data_ptr())
         h = C.c_void_p()

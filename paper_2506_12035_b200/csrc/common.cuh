@@ -2,22 +2,31 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 typedef __nv_bfloat16 bf16;
+typedef __half f16;
 
 #define MARCHE_DEVINL __device__ __forceinline__
 
 MARCHE_DEVINL float to_float(float v) { return v; }
 MARCHE_DEVINL float to_float(bf16 v) { return __bfloat162float(v); }
+MARCHE_DEVINL float to_float(f16 v) { return __half2float(v); }
 
 template <typename T> MARCHE_DEVINL T from_float(float v);
 template <> MARCHE_DEVINL float from_float<float>(float v) { return v; }
 template <> MARCHE_DEVINL bf16 from_float<bf16>(float v) { return __float2bfloat16_rn(v); }
+template <> MARCHE_DEVINL f16 from_float<f16>(float v) { return __float2half_rn(v); }
 
 MARCHE_DEVINL uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+
+MARCHE_DEVINL uint32_t pack_f16x2(float lo, float hi) {
+  __half2 p = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&p);
 }
 
@@ -62,6 +71,12 @@ MARCHE_DEVINL float gelu_erf_fast(float x) {
 // Stores 4 consecutive outputs of type T starting at a 4-element aligned column.
 MARCHE_DEVINL void store4(float* p, float a, float b, float c, float d) {
   *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
+}
+MARCHE_DEVINL void store4(f16* p, float a, float b, float c, float d) {
+  uint2 u;
+  u.x = pack_f16x2(a, b);
+  u.y = pack_f16x2(c, d);
+  *reinterpret_cast<uint2*>(p) = u;
 }
 MARCHE_DEVINL void store4(bf16* p, float a, float b, float c, float d) {
   uint2 u;

@@ -5,7 +5,7 @@
 // to global memory (rows beyond M are clipped by the tensor map).
 //   EPI 0: out bf16 = acc + bias
 //   EPI 1: out fp32 += acc + bias   -- TMA reduce-add in L2, no read in the SM, one add per element
-//   EPI 2: out bf16 = GELU_erf(acc + bias)
+//   EPI 2: out fp16 = GELU_erf(acc + bias)   (feeds the next projection as its A operand)
 #pragma once
 
 #include "sm100_ptx.cuh"
@@ -52,8 +52,10 @@ MARCHE_DEVINL void epilogue_box(uint32_t t_addr, const float* __restrict__ bias_
           v4 = gelu_erf_fast(v4); v5 = gelu_erf_fast(v5); v6 = gelu_erf_fast(v6); v7 = gelu_erf_fast(v7);
         }
         const uint32_t dst = row_base + (uint32_t)(((hh * 4 + j) ^ (lane & 7)) << 4);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pack_bf16x2(v0, v1)),
-                     "r"(pack_bf16x2(v2, v3)), "r"(pack_bf16x2(v4, v5)), "r"(pack_bf16x2(v6, v7)) : "memory");
+        uint32_t p0, p1, p2, p3;
+        if (EPI == 2) { p0 = pack_f16x2(v0, v1); p1 = pack_f16x2(v2, v3); p2 = pack_f16x2(v4, v5); p3 = pack_f16x2(v6, v7); }
+        else { p0 = pack_bf16x2(v0, v1); p1 = pack_bf16x2(v2, v3); p2 = pack_bf16x2(v4, v5); p3 = pack_bf16x2(v6, v7); }
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(p0), "r"(p1), "r"(p2), "r"(p3) : "memory");
       }
     }
   }

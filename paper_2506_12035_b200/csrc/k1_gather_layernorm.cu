@@ -1,6 +1,6 @@
 // K1: index gather + LayerNorm (Algorithm 1 line 5, input side of the QKV and MLP
 // projections).  HBM-bound: each fp32 row is read once with 128-bit loads, kept in
-// registers for the two statistics passes, and written once as T (and, at block 0,
+// registers for the two statistics passes, and written once as fp32 or fp16 (and, at block 0,
 // once more as the compact fp32 residual row).
 //
 // One warp per row: lane l holds float4 number l, l+32, ... of the row (NV per lane),
@@ -82,12 +82,12 @@ static cudaError_t launch_ln_t(const float* src, int src_rows, const int32_t* id
   return cudaGetLastError();
 }
 
-cudaError_t launch_gather_layernorm(bool bf16_out, const float* src, int src_rows, const int32_t* idx,
+cudaError_t launch_gather_layernorm(bool half_out, const float* src, int src_rows, const int32_t* idx,
                                     int B, int n, int D, const float* gamma, const float* beta, float eps,
                                     float* x_out, void* u_out, cudaStream_t st) {
   if (D % 128 != 0) return cudaErrorInvalidValue;
-  if (bf16_out)
-    return launch_ln_t<bf16>(src, src_rows, idx, B, n, D, gamma, beta, eps, x_out, (bf16*)u_out, st);
+  if (half_out)
+    return launch_ln_t<f16>(src, src_rows, idx, B, n, D, gamma, beta, eps, x_out, (f16*)u_out, st);
   return launch_ln_t<float>(src, src_rows, idx, B, n, D, gamma, beta, eps, x_out, (float*)u_out, st);
 }
 

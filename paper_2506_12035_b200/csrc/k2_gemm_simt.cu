@@ -1,5 +1,7 @@
 // K2 (SIMT): out = epilogue(a * w^T + bias) with fp32 FMA arithmetic.
 //
+// Operand types: fp32 x fp32, or (16-bit mode) fp16 activations x fp16 weights; the bias
+// epilogue writes T (fp32 / bf16: q, k, v), the GELU epilogue the activation type (fp32 / fp16).
 // This is the projection kernel of the fp32 configuration (the tensor cores have no
 // full-fp32 mode, and TF32 would not meet an fp32-level tolerance) and the bring-up
 // reference for the bf16 tensor-core kernel.  Classic shared-memory tiling: 64x64
@@ -9,9 +11,9 @@
 
 namespace marche {
 
-template <typename T, int EPI>
+template <typename TA, typename TO, int EPI>
 __global__ void __launch_bounds__(256)
-gemm_simt_kernel(const T* __restrict__ a, int lda, int M, const T* __restrict__ w, const float* __restrict__ bias,
+gemm_simt_kernel(const TA* __restrict__ a, int lda, int M, const TA* __restrict__ w, const float* __restrict__ bias,
                  int N, int K, void* __restrict__ out_) {
   constexpr int BM = 64, BN = 64, BK = 16;
   __shared__ float As[BK][BM + 4];
@@ -70,19 +72,20 @@ gemm_simt_kernel(const T* __restrict__ a, int lda, int M, const T* __restrict__ 
       *p = o;
     } else {
       if (EPI == 2) { v0 = gelu_erf(v0); v1 = gelu_erf(v1); v2 = gelu_erf(v2); v3 = gelu_erf(v3); }
-      store4(reinterpret_cast<T*>(out_) + (long)row * N + col, v0, v1, v2, v3);
+      if (EPI == 2) store4(reinterpret_cast<TA*>(out_) + (long)row * N + col, v0, v1, v2, v3);
+      else store4(reinterpret_cast<TO*>(out_) + (long)row * N + col, v0, v1, v2, v3);
     }
   }
 }
 
-template <typename T>
-static cudaError_t launch_t(const T* a, int lda, int M, const T* w, const float* bias, int N, int K, int epi,
+template <typename TA, typename TO>
+static cudaError_t launch_t(const TA* a, int lda, int M, const TA* w, const float* bias, int N, int K, int epi,
                             void* out, cudaStream_t st) {
   dim3 grid(N / 64, (M + 63) / 64);
   switch (epi) {
-    case 0: gemm_simt_kernel<T, 0><<<grid, 256, 0, st>>>(a, lda, M, w, bias, N, K, out); break;
-    case 1: gemm_simt_kernel<T, 1><<<grid, 256, 0, st>>>(a, lda, M, w, bias, N, K, out); break;
-    case 2: gemm_simt_kernel<T, 2><<<grid, 256, 0, st>>>(a, lda, M, w, bias, N, K, out); break;
+    case 0: gemm_simt_kernel<TA, TO, 0><<<grid, 256, 0, st>>>(a, lda, M, w, bias, N, K, out); break;
+    case 1: gemm_simt_kernel<TA, TO, 1><<<grid, 256, 0, st>>>(a, lda, M, w, bias, N, K, out); break;
+    case 2: gemm_simt_kernel<TA, TO, 2><<<grid, 256, 0, st>>>(a, lda, M, w, bias, N, K, out); break;
     default: return cudaErrorInvalidValue;
   }
   return cudaGetLastError();
@@ -92,8 +95,8 @@ cudaError_t launch_gemm_simt(bool bf16_t, const void* a, int lda, int M, const v
                              int N, int K, int epilogue, void* out, cudaStream_t st) {
   if (M == 0) return cudaSuccess;
   if (N % 64 || K % 16) return cudaErrorInvalidValue;
-  if (bf16_t) return launch_t<bf16>((const bf16*)a, lda, M, (const bf16*)w, bias, N, K, epilogue, out, st);
-  return launch_t<float>((const float*)a, lda, M, (const float*)w, bias, N, K, epilogue, out, st);
+  if (bf16_t) return launch_t<f16, bf16>((const f16*)a, lda, M, (const f16*)w, bias, N, K, epilogue, out, st);
+  return launch_t<float, float>((const float*)a, lda, M, (const float*)w, bias, N, K, epilogue, out, st);
 }
 
 }  // namespace marche

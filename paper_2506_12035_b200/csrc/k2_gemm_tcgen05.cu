@@ -1,11 +1,11 @@
 // K2: out = epilogue(a * w^T + bias) on the 5th-generation tensor cores.
 //
 // The QKV, output and MLP projections of the active rows (Algorithm 1 lines 5 and 9)
-// are dense bf16 contractions, so they run as a persistent, warp-specialised tcgen05
+// are dense 16-bit contractions (fp16 activations x fp16 weights -> fp32), so they run as a persistent, warp-specialised tcgen05
 // kernel: one CTA per SM walks over 128 x BN output tiles;
 //   warp 0   (one lane)  TMA producer: 128x64 A tile and BNx64 W tile per K step into a
 //                        shared-memory ring (128-byte swizzle), completion on mbarriers
-//   warp 1   (one lane)  issues tcgen05.mma (M 128, N BN, K 16; bf16 in, fp32 accumulate
+//   warp 1   (one lane)  issues tcgen05.mma (M 128, N BN, K 16; fp16 in, fp32 accumulate
 //                        in TMEM), frees ring slots and publishes accumulators with
 //                        tcgen05.commit
 //   warps 2-5            epilogue: tcgen05.ld of the accumulator (thread = output row),
@@ -121,7 +121,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = ptx::idesc_bf16_f32(BM, BN);
+      constexpr uint32_t idesc = ptx::idesc_f16_f32(BM, BN);
       int it = 0, tile_i = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tile_i) {
@@ -186,11 +186,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
 
 // ---------------------------------------------------------------- host side
 // Row-major bf16 matrix [rows][cols] with row stride ld elements; box = 64 columns x box_rows rows.
-bool make_map_2d(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
+bool make_map_2d(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows,
+                 bool ieee_half) {
   const uint64_t dims[2] = {cols, rows};
   const uint64_t strides[1] = {ld * 2};
   const uint32_t box[2] = {BK, box_rows};
-  return tma_make_map_bf16(map, ptr, 2, dims, strides, box, true);
+  return tma_make_map_bf16(map, ptr, 2, dims, strides, box, true, ieee_half);
 }
 
 int sm_count() { return device_sm_count(); }
@@ -228,8 +229,8 @@ cudaError_t launch_gemm_tcgen05(const void* a, int lda, int M, const void* w, co
   if (N % 128 || K % BK || lda % 8 || ((uintptr_t)a & 15) || ((uintptr_t)w & 15)) return cudaErrorInvalidValue;
   const int bn = gemm_tcgen05_pick_bn(M, N);
   CUtensorMap ta, tw, to;
-  if (!make_map_2d(&ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM)) return cudaErrorInvalidValue;
-  if (!make_map_2d(&tw, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)bn)) return cudaErrorInvalidValue;
+  if (!make_map_2d(&ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM, true)) return cudaErrorInvalidValue;
+  if (!make_map_2d(&tw, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)bn, true)) return cudaErrorInvalidValue;
   if (((uintptr_t)out & 15) || !tma_make_store_map(&to, out, (uint64_t)M, (uint64_t)N, epilogue == 1 ? 4 : 2))
     return cudaErrorInvalidValue;
 #define MARCHE_GEMM_CASE(BN_, EPI_) \

@@ -125,7 +125,7 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer (leader only)
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = ptx::idesc_bf16_f32(2 * BM, BN);
+      constexpr uint32_t idesc = ptx::idesc_f16_f32(2 * BM, BN);
       int it = 0, tile_i = 0;
       bool ok = true;
       for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++tile_i) {
@@ -190,11 +190,12 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
   }
 }
 
-bool make_map_2d(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
+bool make_map_2d(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows,
+                 bool ieee_half) {
   const uint64_t dims[2] = {cols, rows};
   const uint64_t strides[1] = {ld * 2};
   const uint32_t box[2] = {BK, box_rows};
-  return tma_make_map_bf16(map, ptr, 2, dims, strides, box, true);
+  return tma_make_map_bf16(map, ptr, 2, dims, strides, box, true, ieee_half);
 }
 
 template <int BN, int EPI>
@@ -237,8 +238,8 @@ cudaError_t launch_gemm_tcgen05_2cta(const void* a, int lda, int M, const void* 
   if (N % 128 || K % BK || lda % 8 || ((uintptr_t)a & 15) || ((uintptr_t)w & 15)) return cudaErrorInvalidValue;
   const int bn = gemm_tcgen05_2cta_pick_bn(M, N);
   CUtensorMap ta, tw, to;
-  if (!make_map_2d(&ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM)) return cudaErrorInvalidValue;
-  if (!make_map_2d(&tw, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)(bn / 2))) return cudaErrorInvalidValue;
+  if (!make_map_2d(&ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM, true)) return cudaErrorInvalidValue;
+  if (!make_map_2d(&tw, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)(bn / 2), true)) return cudaErrorInvalidValue;
   if (((uintptr_t)out & 15) || !tma_make_store_map(&to, out, (uint64_t)M, (uint64_t)N, epilogue == 1 ? 4 : 2))
     return cudaErrorInvalidValue;
 #define MARCHE_GEMM2_CASE(BN_, EPI_) \

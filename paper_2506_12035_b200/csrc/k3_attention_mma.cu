@@ -9,7 +9,8 @@
 // through a 3-deep shared-memory ring (128-byte swizzle for head_dim 64) straight from
 // the token-major cache [2][B][S][D]; several CTAs are resident per SM.  QK^T and PV
 // run on the tensor cores (mma.sync m16n8k16, bf16 in, fp32 accumulate; each warp owns
-// 16 query rows), softmax statistics stay in fp32 registers.
+// 16 query rows), softmax statistics stay in fp32 registers.  The output rows are written
+// as fp16: they are the A operand of the output projection.
 //
 // Two flavours:
 //   plain    one pass, online softmax (running max / sum, rescaled accumulators);
@@ -67,7 +68,7 @@ template <int DH, int NWARPS, bool SCORING>
 __global__ void __launch_bounds__(NWARPS * 32)
 attention_mma_kernel(const __grid_constant__ CUtensorMap tmap_kv, const bf16* __restrict__ q, int ld_q, int n,
                      int S, int H, int B, const uint8_t* __restrict__ is_new, float* __restrict__ score_partial,
-                     bf16* __restrict__ o, int* __restrict__ status) {
+                     f16* __restrict__ o, int* __restrict__ status) {
   using Cfg = AttCfg<DH>;
   constexpr int QT = NWARPS * 16;
   extern __shared__ uint8_t smem_raw[];
@@ -279,12 +280,12 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap tmap_kv, const bf16* __
       if (final_pass && kt == n_kv - 1) {
         const float f0 = SCORING ? 1.0f : 1.0f / l_run[0], f1 = SCORING ? 1.0f : 1.0f / l_run[1];
         const int r0 = qt * QT + warp * 16 + g, r1 = r0 + 8;
-        bf16* o0 = o + ((size_t)b * n + r0) * D + h * DH + 2 * tg;
-        bf16* o1 = o + ((size_t)b * n + r1) * D + h * DH + 2 * tg;
+        f16* o0 = o + ((size_t)b * n + r0) * D + h * DH + 2 * tg;
+        f16* o1 = o + ((size_t)b * n + r1) * D + h * DH + 2 * tg;
 #pragma unroll
         for (int j = 0; j < Cfg::ONT; ++j) {
-          if (r0 < n) *reinterpret_cast<uint32_t*>(o0 + 8 * j) = pack_bf16x2(oacc[j][0] * f0, oacc[j][1] * f0);
-          if (r1 < n) *reinterpret_cast<uint32_t*>(o1 + 8 * j) = pack_bf16x2(oacc[j][2] * f1, oacc[j][3] * f1);
+          if (r0 < n) *reinterpret_cast<uint32_t*>(o0 + 8 * j) = pack_f16x2(oacc[j][0] * f0, oacc[j][1] * f0);
+          if (r1 < n) *reinterpret_cast<uint32_t*>(o1 + 8 * j) = pack_f16x2(oacc[j][2] * f1, oacc[j][3] * f1);
         }
       }
     }
@@ -315,7 +316,7 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap tmap_kv, const bf16* __
 
 template <int DH, int NWARPS, bool SCORING>
 cudaError_t launch_att(const CUtensorMap& tm, const bf16* q, int ld_q, int B, int n, int S, int H,
-                       const uint8_t* is_new, float* partial, bf16* o, int* status, cudaStream_t st) {
+                       const uint8_t* is_new, float* partial, f16* o, int* status, cudaStream_t st) {
   const size_t smem = NSTAGE * AttCfg<DH>::STAGE_BYTES + 1024 + 64 + (SCORING ? (size_t)NWARPS * S * sizeof(float) : 0);
   static size_t smem_set = 0;
   if (smem > smem_set) {
@@ -331,7 +332,7 @@ cudaError_t launch_att(const CUtensorMap& tm, const bf16* q, int ld_q, int B, in
 
 template <int DH>
 cudaError_t launch_dh(const CUtensorMap& tm, const bf16* q, int ld_q, int B, int n, int S, int H,
-                      const uint8_t* is_new, float* partial, bf16* o, int* status, cudaStream_t st) {
+                      const uint8_t* is_new, float* partial, f16* o, int* status, cudaStream_t st) {
   const bool sc = is_new != nullptr;
   const int nw = n <= 32 ? 2 : (n <= 64 ? 4 : 8);
 #define MARCHE_ATT_CASE(NW_)                                                                              \
@@ -358,8 +359,8 @@ cudaError_t launch_attention_mma(const void* q, int ld_q, int B, int n, int S, i
   const uint32_t box[3] = {(uint32_t)dh, KT, 1};
   if (!tma_make_map_bf16(&tm, cache_layer, 3, dims, strides, box, dh == 64)) return cudaErrorInvalidValue;
   if (dh == 64)
-    return launch_dh<64>(tm, (const bf16*)q, ld_q, B, n, S, H, is_new, score_partial, (bf16*)o, status, st);
-  return launch_dh<80>(tm, (const bf16*)q, ld_q, B, n, S, H, is_new, score_partial, (bf16*)o, status, st);
+    return launch_dh<64>(tm, (const bf16*)q, ld_q, B, n, S, H, is_new, score_partial, (f16*)o, status, st);
+  return launch_dh<80>(tm, (const bf16*)q, ld_q, B, n, S, H, is_new, score_partial, (f16*)o, status, st);
 }
 
 }  // namespace marche

@@ -19,11 +19,11 @@ size_t attention_simt_smem(int S, int dh) {
   return (size_t)kAttWarps * (2 * (size_t)S + dh) * sizeof(float);
 }
 
-template <typename T>
+template <typename T, typename TO>
 __global__ void __launch_bounds__(kAttWarps * 32)
 attention_simt_kernel(const T* __restrict__ q, int ld_q, int n, int S, int H, int dh,
                       const T* __restrict__ cache_layer, long kv_stride, const uint8_t* __restrict__ is_new,
-                      float* __restrict__ score_partial, T* __restrict__ o) {
+                      float* __restrict__ score_partial, TO* __restrict__ o) {
   extern __shared__ float smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.x / H, h = blockIdx.x % H;
@@ -70,7 +70,7 @@ attention_simt_kernel(const T* __restrict__ q, int ld_q, int n, int S, int H, in
     for (int c = lane; c < dh; c += 32) {
       float acc = 0.f;
       for (int t = 0; t < S; ++t) acc = fmaf(p[t], to_float(Vb[(long)t * D + c]), acc);
-      o[r * D + h * dh + c] = from_float<T>(acc);
+      o[r * D + h * dh + c] = from_float<TO>(acc);
     }
   }
   if (scoring) {
@@ -91,14 +91,14 @@ cudaError_t launch_attention_simt(bool bf16_t, const void* q, int ld_q, int B, i
   const long kv_stride = (long)B * S * H * dh;
   cudaError_t e;
   if (bf16_t) {
-    e = cudaFuncSetAttribute(attention_simt_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(attention_simt_kernel<bf16, f16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attention_simt_kernel<bf16><<<B * H, kAttWarps * 32, smem, st>>>(
-        (const bf16*)q, ld_q, n, S, H, dh, (const bf16*)cache_layer, kv_stride, is_new, score_partial, (bf16*)o);
+    attention_simt_kernel<bf16, f16><<<B * H, kAttWarps * 32, smem, st>>>(
+        (const bf16*)q, ld_q, n, S, H, dh, (const bf16*)cache_layer, kv_stride, is_new, score_partial, (f16*)o);
   } else {
-    e = cudaFuncSetAttribute(attention_simt_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(attention_simt_kernel<float, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attention_simt_kernel<float><<<B * H, kAttWarps * 32, smem, st>>>(
+    attention_simt_kernel<float, float><<<B * H, kAttWarps * 32, smem, st>>>(
         (const float*)q, ld_q, n, S, H, dh, (const float*)cache_layer, kv_stride, is_new, score_partial, (float*)o);
   }
   return cudaGetLastError();

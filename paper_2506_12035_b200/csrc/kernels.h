@@ -8,8 +8,8 @@
 
 namespace marche {
 
-// K1: gather + LayerNorm.  rows = B*n; src row of (b, j) is src[b][idx ? idx[b][j] : j].
-cudaError_t launch_gather_layernorm(bool bf16_out, const float* src, int src_rows, const int32_t* idx,
+// K1: gather + LayerNorm (output fp16 when half_out, else fp32).  rows = B*n; src row of (b, j) is src[b][idx ? idx[b][j] : j].
+cudaError_t launch_gather_layernorm(bool half_out, const float* src, int src_rows, const int32_t* idx,
                                     int B, int n, int D, const float* gamma, const float* beta, float eps,
                                     float* x_out, void* u_out, cudaStream_t st);
 

@@ -27,10 +27,11 @@ inline EncodeTiledFn tma_encode_fn() {
   return fn;
 }
 
-// bf16 tensor of `rank` dimensions (innermost first).  strides_bytes has rank-1 entries
+// 16-bit (bf16, or fp16 when ieee_half) tensor of `rank` dimensions (innermost first).  strides_bytes has rank-1 entries
 // (the innermost stride is the element size).  Out-of-bounds elements read as zero.
 inline bool tma_make_map_bf16(CUtensorMap* map, const void* ptr, int rank, const uint64_t* dims,
-                              const uint64_t* strides_bytes, const uint32_t* box, bool swizzle128) {
+                              const uint64_t* strides_bytes, const uint32_t* box, bool swizzle128,
+                              bool ieee_half = false) {
   EncodeTiledFn fn = tma_encode_fn();
   if (!fn) return false;
   cuuint64_t d[5], s[5];
@@ -41,7 +42,8 @@ inline bool tma_make_map_bf16(CUtensorMap* map, const void* ptr, int rank, const
     e[i] = 1;
     if (i + 1 < rank) s[i] = strides_bytes[i];
   }
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(ptr), d, s, b, e,
+  return fn(map, ieee_half ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank,
+            const_cast<void*>(ptr), d, s, b, e,
             CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }

@@ -149,7 +149,7 @@ def make_weights(cfg: MarConfig, seed: int = SEED_WEIGHTS, n_blocks: int | None 
                  ) -> List[Dict[str, np.ndarray]]:
     """Per block: fp32 arrays.  Linear weights ([out][in]) and all biases
     ~ N(0, 0.02^2); LayerNorm gain 1 + N(0, 0.02^2), shift N(0, 0.02^2).
-    For bf16 configs the four matrices are rounded to bf16-representable values."""
+    For bf16 configs the four matrices are rounded to values that both bf16 and fp16 hold exactly."""
     rng = np.random.Generator(np.random.Philox(seed))
     D, F = cfg.D, cfg.F
     shapes = {
@@ -165,7 +165,8 @@ def make_weights(cfg: MarConfig, seed: int = SEED_WEIGHTS, n_blocks: int | None 
             if name in ("ln1_g", "ln2_g"):
                 a = a + np.float32(1.0)
             if cfg.dtype == "bf16" and name in MATRIX_FIELDS:
-                a = round_to_bf16(a)
+                # representable in bf16 and in fp16, so any 16-bit copy of it is exact
+                a = round_to_bf16(a).astype(np.float16).astype(np.float32)
             blk[name] = np.ascontiguousarray(a, dtype=np.float32)
         blocks.append(blk)
     return blocks

@@ -1,0 +1,92 @@
+"""Parity at the benchmark's full size, in the launch configuration bench.py times: the
+MAR-L-shaped stack (32 blocks, width 1024, 16 heads, S 320) at batch 128.  The GPU runs the
+whole batch; the oracle runs one classifier-free-guidance pair (rows 0 and 64) - samples are
+independent (pinned by the oracle's sample-independence test), so their rows must match the
+oracle's.  One full step and two cache-aware steps, teacher-forced with the oracle's refresh
+sets for the pair (the other rows use the device's own selection)."""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import marche_oracle as orc
+from helpers import TOL, dev, idx_dev, make_model, max_abs, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name", ["mar_l"])
+def test_full_size_sampled_parity(name):
+    cfg = synth.CONFIGS[name]
+    if torch.cuda.get_device_properties(0).total_memory < 40e9:
+        pytest.skip("needs a large GPU")
+    pair = [0, cfg.B // 2]
+    ratio, n_steps = cfg.ratio, 3
+    blocks = synth.make_weights(cfg)
+    m = make_model(cfg, blocks)
+    hidden_np = synth.make_hidden(cfg)
+    sets = synth.new_token_sets(cfg, synth.generation_orders(cfg))
+
+    # ---- oracle on the pair
+    h2 = hidden_np[pair].copy()
+    s2 = [g[pair] for g in sets]
+    cache2 = orc.KVCache(cfg.L, 2, cfg.S, cfg.D)
+    out2 = np.zeros_like(h2)
+    kw = dict(n_heads=cfg.H, score_layer=cfg.score_layer, ln_eps=cfg.ln_eps)
+    recs = []
+    sc, R = orc.full_step(blocks, h2, cache2, s2[0], s2[1], ratio, out2, **kw)
+    recs.append(dict(active=np.tile(np.arange(cfg.S, dtype=np.int32), (2, 1)), out=out2.copy(), scores=sc, refresh=R))
+    for t in range(1, n_steps):
+        rows = synth.replacement_rows(cfg, t - 1, s2[t - 1].shape[1], batch=cfg.B)[pair]
+        for i in range(2):
+            h2[i, s2[t - 1][i]] = rows[i]
+        A = orc.active_set(s2[t], s2[t - 1], R)
+        sc, R = orc.marche_step(blocks, h2, cache2, A, s2[t], s2[t + 1], ratio, out2, **kw)
+        recs.append(dict(active=A, out=out2.copy(), scores=sc, refresh=R))
+    del blocks
+
+    # ---- device on the whole batch
+    B, S, D = cfg.B, cfg.S, cfg.D
+    hidden = dev(hidden_np)
+    hidden_out = torch.zeros(B, S, D, device="cuda")
+    cache = m.alloc_cache()
+    ws = m.alloc_workspace(S)
+    m.init_cache(cache)
+    refresh = torch.zeros(B * S, dtype=torch.int32, device="cuda")
+    scores = torch.empty(B, S, device="cuda")
+    ma, rl = TOL["bf16"]
+    k_prev = 0
+    worst = 0.0
+    for t in range(n_steps):
+        G, X = idx_dev(sets[t]), idx_dev(sets[t + 1])
+        if t == 0:
+            k = m.full_step(hidden, cache, G, X, ratio, hidden_out, refresh, ws)
+        else:
+            m.scatter_rows(dev(synth.replacement_rows(cfg, t - 1, sets[t - 1].shape[1])), idx_dev(sets[t - 1]), hidden)
+            nA = sets[t].shape[1] + sets[t - 1].shape[1] + k_prev
+            active = torch.empty(B, nA, dtype=torch.int32, device="cuda")
+            m.build_active(G, idx_dev(sets[t - 1]), refresh, k_prev, active)
+            assert np.array_equal(active[pair].cpu().numpy(), recs[t]["active"])
+            k = m.step(hidden, cache, active, G, X, ratio, hidden_out, refresh, ws)
+        m.get_scores(ws, scores)
+        torch.cuda.synchronize()
+        assert m.device_status() == 0
+        rec = recs[t]
+        assert k == rec["refresh"].shape[1]
+        got = hidden_out[pair].cpu().numpy()
+        for i in range(2):
+            a, w = got[i, rec["active"][i]], rec["out"][i, rec["active"][i]]
+            worst = max(worst, max_abs(a, w))
+            assert max_abs(a, w) <= ma and rel_l2(a, w) <= rl, \
+                "step %d sample %d: max-abs %.3g rel-L2 %.3g" % (t, pair[i], max_abs(a, w), rel_l2(a, w))
+        unit = cfg.H * sets[t].shape[1] / cfg.S
+        assert max_abs(scores[pair].cpu().numpy(), rec["scores"]) <= 5e-2 * unit
+        # teacher forcing: the pair continues with the oracle's refresh set
+        r = refresh[: B * k].view(B, k)
+        r[pair] = torch.as_tensor(rec["refresh"]).cuda()
+        k_prev = k
+    Kc = cache[:, 0][:, pair].float().cpu().numpy()
+    Vc = cache[:, 1][:, pair].float().cpu().numpy()
+    assert max_abs(Kc, cache2.K) <= ma and rel_l2(Kc, cache2.K) <= rl
+    assert max_abs(Vc, cache2.V) <= ma and rel_l2(Vc, cache2.V) <= rl
+    print("full-size parity: hidden max-abs %.3g, cache K max-abs %.3g" % (worst, max_abs(Kc, cache2.K)))

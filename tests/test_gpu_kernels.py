@@ -20,7 +20,17 @@ def model_for(dtype, D, H, F, S, B, L=1):
 
 
 def tdt(dtype):
+    """element type of weights, q/k/v and the K/V cache"""
     return torch.bfloat16 if dtype == "bf16" else torch.float32
+
+
+def adt(dtype):
+    """element type of the activation matrices that feed a projection (fp16 in 16-bit mode)"""
+    return torch.float16 if dtype == "bf16" else torch.float32
+
+
+def quant_a(a, dtype):
+    return np.asarray(a, np.float32).astype(np.float16).astype(np.float64) if dtype == "bf16" else np.asarray(a, np.float32).astype(np.float64)
 
 
 def quant(a, dtype):
@@ -43,14 +53,14 @@ def test_gather_layernorm(dtype, D, H, n):
     g, be = blocks[0]["ln1_g"], blocks[0]["ln1_b"]
     for idx in patterns:
         x_out = torch.full((B * n, D), -7.0, device="cuda")
-        u_out = torch.zeros(B * n, D, dtype=tdt(dtype), device="cuda")
+        u_out = torch.zeros(B * n, D, dtype=adt(dtype), device="cuda")
         m.gather_layernorm(dev(hidden), idx_dev(idx), n, dev(g), dev(be), x_out, u_out)
         X = np.stack([hidden[b, idx[b]] for b in range(B)]).reshape(B * n, D)
         assert np.array_equal(x_out.cpu().numpy(), X)                       # the gather is a copy: exact
         want = orc.layer_norm(X.astype(np.float64), g.astype(np.float64), be.astype(np.float64), cfg.ln_eps)
         assert_close(host(u_out), want, dtype, "LN", scale=1.0 if dtype == "bf16" else 10.0)
     # identity index (idx NULL), no compact copy
-    u_out = torch.zeros(B * n, D, dtype=tdt(dtype), device="cuda")
+    u_out = torch.zeros(B * n, D, dtype=adt(dtype), device="cuda")
     m.gather_layernorm(dev(hidden), None, n, dev(g), dev(be), None, u_out)
     want = orc.layer_norm(hidden[:, :n].reshape(B * n, D).astype(np.float64), g.astype(np.float64),
                           be.astype(np.float64), cfg.ln_eps)
@@ -67,9 +77,9 @@ def test_linear_all_epilogues(dtype, M, N, K):
     a = rng.standard_normal((M, K)).astype(np.float32)
     w = (rng.standard_normal((N, K)) * 0.05).astype(np.float32)
     bias = rng.standard_normal(N).astype(np.float32)
-    aq, wq = quant(a, dtype), quant(w, dtype)
+    aq, wq = quant_a(a, dtype), quant_a(w, dtype)
     acc = orc.linear(aq, wq, bias.astype(np.float64))
-    a_d, w_d, b_d = dev(a, tdt(dtype)), dev(w, tdt(dtype)), dev(bias)
+    a_d, w_d, b_d = dev(a, adt(dtype)), dev(w, adt(dtype)), dev(bias)
     ma, rl = TOL[dtype]
     # bias
     out = torch.zeros(M, N, dtype=tdt(dtype), device="cuda")
@@ -82,7 +92,7 @@ def test_linear_all_epilogues(dtype, M, N, K):
     m.linear(a_d, w_d, b_d, 1, out)
     assert max_abs(host(out), acc + res) <= 1e-4 * max(1.0, math.sqrt(K / 256))
     # bias + GELU
-    out = torch.zeros(M, N, dtype=tdt(dtype), device="cuda")
+    out = torch.zeros(M, N, dtype=adt(dtype), device="cuda")
     m.linear(a_d, w_d, b_d, 2, out)
     want = orc.gelu(acc)
     assert rel_l2(host(out), want) <= (4e-3 if dtype == "bf16" else 1e-6)
@@ -98,10 +108,10 @@ def test_linear_strided_input_and_row_guard(dtype):
     wide = rng.standard_normal((M, 3 * K)).astype(np.float32)
     w = (rng.standard_normal((N, K)) * 0.05).astype(np.float32)
     bias = rng.standard_normal(N).astype(np.float32)
-    wide_d = dev(wide, tdt(dtype))
+    wide_d = dev(wide, adt(dtype))
     out = torch.full((M + 60, N), 5.0, dtype=tdt(dtype), device="cuda")
-    m.linear(wide_d[:, K:2 * K], dev(w, tdt(dtype)), dev(bias), 0, out, M=M, lda=3 * K)
-    want = orc.linear(quant(wide[:, K:2 * K], dtype), quant(w, dtype), bias.astype(np.float64))
+    m.linear(wide_d[:, K:2 * K], dev(w, adt(dtype)), dev(bias), 0, out, M=M, lda=3 * K)
+    want = orc.linear(quant_a(wide[:, K:2 * K], dtype), quant_a(w, dtype), bias.astype(np.float64))
     assert rel_l2(host(out[:M]), want) <= (4e-3 if dtype == "bf16" else 1e-6)
     assert (host(out[M:]) == 5.0).all()
 
@@ -169,7 +179,7 @@ def test_attention_and_score_partials(dtype, S, dh, H, n, nG):
     for b in range(B):
         flags[b, rng.permutation(n)[:nG]] = 1
     q_d = dev(q, tdt(dtype))
-    o = torch.zeros(B * n, D, dtype=tdt(dtype), device="cuda")
+    o = torch.zeros(B * n, D, dtype=adt(dtype), device="cuda")
     partial = torch.full((B, H, S), -1.0, device="cuda")
     m.attention(q_d, 3 * D, n, dev(cache, tdt(dtype)), dev(flags), partial, o)
     qq, cc = quant(q, dtype), quant(cache, dtype)
@@ -201,7 +211,7 @@ def test_attention_uniform_and_peaked(dtype):
     cache = rng.standard_normal((2, B, S, D)).astype(np.float32)
     flags = np.ones((B, n), dtype=np.uint8)
     # q = 0 -> uniform weights: o = mean of V, partial = n / S
-    o = torch.zeros(B * n, D, dtype=tdt(dtype), device="cuda")
+    o = torch.zeros(B * n, D, dtype=adt(dtype), device="cuda")
     partial = torch.zeros(B, H, S, device="cuda")
     m.attention(torch.zeros(B * n, D, dtype=tdt(dtype), device="cuda"), D, n, dev(cache, tdt(dtype)), dev(flags),
                 partial, o)
