@@ -265,7 +265,7 @@ def run_ours(args, cfg):
 
     line = {"metric": METRIC, "value": value, "unit": "images/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_gen, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+            "vs_baseline": None, "dtype": "fp16 projections + bf16 attention/cache, fp32 accumulate" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
             "config": workload_config(cfg, ratio), "clocks": clock_info, "gpu_launches": int(launches),
             "ms_per_decoding_step": ms_gen / cfg.T}
 

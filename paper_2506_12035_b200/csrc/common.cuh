@@ -35,6 +35,15 @@ MARCHE_DEVINL float2 unpack_bf16x2(uint32_t u) {
   return __bfloat1622float2(p);
 }
 
+// Programmatic dependent launch: wait for the preceding kernel of the stream (no-op when the
+// launch did not opt in), then allow the following kernel to start launching.
+MARCHE_DEVINL void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+MARCHE_DEVINL void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+MARCHE_DEVINL void pdl_sync() {
+  pdl_wait();
+  pdl_launch_dependents();
+}
+
 MARCHE_DEVINL float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

@@ -7,6 +7,7 @@
 // so every load/store instruction of a warp covers 512 contiguous bytes.
 #include "common.cuh"
 #include "kernels.h"
+#include "launch_pdl.h"
 
 namespace marche {
 
@@ -22,6 +23,7 @@ gather_layernorm_kernel(const float* __restrict__ src, int src_rows, const int32
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long r = (long)blockIdx.x * kLnWarps + warp;
   if (r >= total_rows) return;
+  pdl_sync();
   const int b = (int)(r / n), j = (int)(r - (long)b * n);
   const int srow = idx ? idx[r] : j;
   const float4* __restrict__ in = reinterpret_cast<const float4*>(src + ((long)b * src_rows + srow) * D);
@@ -66,10 +68,11 @@ static cudaError_t launch_ln_t(const float* src, int src_rows, const int32_t* id
   const long rows = (long)B * n;
   if (rows == 0) return cudaSuccess;
   const unsigned grid = (unsigned)((rows + kLnWarps - 1) / kLnWarps);
+  cudaError_t err = cudaSuccess;
 #define MARCHE_LN_CASE(NV_)                                                                          \
   case NV_:                                                                                          \
-    gather_layernorm_kernel<TOut, NV_><<<grid, kLnWarps * 32, 0, st>>>(src, src_rows, idx, n, (int)rows, \
-                                                                      gamma, beta, eps, x_out, u_out); \
+    err = launch_pdl(gather_layernorm_kernel<TOut, NV_>, dim3(grid), dim3(kLnWarps * 32), 0, st, src, src_rows, \
+                     idx, n, (int)rows, gamma, beta, eps, x_out, u_out);                             \
     break;
   switch (D / 128) {
     MARCHE_LN_CASE(1) MARCHE_LN_CASE(2) MARCHE_LN_CASE(3) MARCHE_LN_CASE(4) MARCHE_LN_CASE(5)
@@ -79,7 +82,7 @@ static cudaError_t launch_ln_t(const float* src, int src_rows, const int32_t* id
     default: return cudaErrorInvalidValue;
   }
 #undef MARCHE_LN_CASE
-  return cudaGetLastError();
+  return err;
 }
 
 cudaError_t launch_gather_layernorm(bool half_out, const float* src, int src_rows, const int32_t* idx,

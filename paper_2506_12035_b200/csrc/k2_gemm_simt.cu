@@ -8,6 +8,7 @@
 // output tile, K step 16, 256 threads each owning a 4x4 micro-tile.
 #include "common.cuh"
 #include "kernels.h"
+#include "launch_pdl.h"
 
 namespace marche {
 
@@ -19,6 +20,7 @@ gemm_simt_kernel(const TA* __restrict__ a, int lda, int M, const TA* __restrict_
   __shared__ float As[BK][BM + 4];
   __shared__ float Ws[BK][BN + 4];
   const int tid = threadIdx.x;
+  pdl_sync();
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
   const int tx = tid & 15, ty = tid >> 4;       // micro-tile origin: rows ty*4, cols tx*4
   const int lr = tid >> 2, lk = (tid & 3) * 4;  // loader: row lr (0..63), k offset lk (0,4,8,12)
@@ -83,12 +85,11 @@ static cudaError_t launch_t(const TA* a, int lda, int M, const TA* w, const floa
                             void* out, cudaStream_t st) {
   dim3 grid(N / 64, (M + 63) / 64);
   switch (epi) {
-    case 0: gemm_simt_kernel<TA, TO, 0><<<grid, 256, 0, st>>>(a, lda, M, w, bias, N, K, out); break;
-    case 1: gemm_simt_kernel<TA, TO, 1><<<grid, 256, 0, st>>>(a, lda, M, w, bias, N, K, out); break;
-    case 2: gemm_simt_kernel<TA, TO, 2><<<grid, 256, 0, st>>>(a, lda, M, w, bias, N, K, out); break;
+    case 0: return launch_pdl(gemm_simt_kernel<TA, TO, 0>, grid, dim3(256), 0, st, a, lda, M, w, bias, N, K, out);
+    case 1: return launch_pdl(gemm_simt_kernel<TA, TO, 1>, grid, dim3(256), 0, st, a, lda, M, w, bias, N, K, out);
+    case 2: return launch_pdl(gemm_simt_kernel<TA, TO, 2>, grid, dim3(256), 0, st, a, lda, M, w, bias, N, K, out);
     default: return cudaErrorInvalidValue;
   }
-  return cudaGetLastError();
 }
 
 cudaError_t launch_gemm_simt(bool bf16_t, const void* a, int lda, int M, const void* w, const float* bias,

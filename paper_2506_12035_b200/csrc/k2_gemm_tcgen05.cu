@@ -19,6 +19,7 @@
 
 #include "gemm_epilogue.cuh"
 #include "kernels.h"
+#include "launch_pdl.h"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"
 
@@ -89,6 +90,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_sync();                                               // set-up above overlaps the previous kernel's tail
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
@@ -208,8 +210,8 @@ cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tw, const CUten
   }
   const int n_tiles = ((M + BM - 1) / BM) * (N / BN);
   const int grid = n_tiles < sm_count() ? n_tiles : sm_count();
-  gemm_tcgen05_kernel<BN, EPI><<<grid, kGemmThreads, GemmCfg<BN>::SMEM_BYTES, st>>>(ta, tw, to, M, N, K, bias, status);
-  return cudaGetLastError();
+  return launch_pdl(gemm_tcgen05_kernel<BN, EPI>, dim3(grid), dim3(kGemmThreads), (size_t)GemmCfg<BN>::SMEM_BYTES, st, ta,
+                    tw, to, M, N, K, bias, status);
 }
 
 }  // namespace

@@ -23,6 +23,7 @@
 
 #include "gemm_epilogue.cuh"
 #include "kernels.h"
+#include "launch_pdl.h"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"
 
@@ -97,6 +98,7 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
   ptx::cluster_sync_all();                                // both CTAs' barriers exist before any remote signal
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_sync();                                             // set-up above overlaps the previous kernel's tail
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer (both CTAs)
@@ -211,9 +213,8 @@ cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUte
   const int n_tiles = ((M + 2 * BM - 1) / (2 * BM)) * (N / BN);
   const int max_pairs = device_sm_count() / 2;
   const int pairs = n_tiles < max_pairs ? n_tiles : max_pairs;
-  gemm_tcgen05_2cta_kernel<BN, EPI><<<2 * pairs, kThreads, PairCfg<BN>::SMEM_BYTES, st>>>(ta, tw, to, M, N, K, bias,
-                                                                                         status);
-  return cudaGetLastError();
+  return launch_pdl(gemm_tcgen05_2cta_kernel<BN, EPI>, dim3(2 * pairs), dim3(kThreads), (size_t)PairCfg<BN>::SMEM_BYTES,
+                    st, ta, tw, to, M, N, K, bias, status);
 }
 
 }  // namespace

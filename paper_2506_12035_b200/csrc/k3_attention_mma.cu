@@ -23,6 +23,7 @@
 #include <cuda.h>
 
 #include "kernels.h"
+#include "launch_pdl.h"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"
 
@@ -98,6 +99,7 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap tmap_kv, const bf16* __
   if (SCORING)
     for (int t = threadIdx.x; t < NWARPS * S; t += NWARPS * 32) colsum[t] = 0.f;
   __syncthreads();
+  pdl_sync();                                          // set-up above overlaps the previous kernel's tail
 
   // Load number i of the CTA's fixed sequence (per q-tile: [K tiles of pass 1,] then K+V tiles).
   auto issue = [&](int i) {
@@ -325,9 +327,8 @@ cudaError_t launch_att(const CUtensorMap& tm, const bf16* q, int ld_q, int B, in
     if (e != cudaSuccess) return e;
     smem_set = smem;
   }
-  attention_mma_kernel<DH, NWARPS, SCORING><<<B * H, NWARPS * 32, smem, st>>>(tm, q, ld_q, n, S, H, B, is_new, partial,
-                                                                             o, status);
-  return cudaGetLastError();
+  return launch_pdl(attention_mma_kernel<DH, NWARPS, SCORING>, dim3(B * H), dim3(NWARPS * 32), smem, st, tm, q, ld_q, n,
+                    S, H, B, is_new, partial, o, status);
 }
 
 template <int DH>

@@ -10,6 +10,7 @@
 // sums and the warps are combined in fixed order: scores are bit-reproducible.
 #include "common.cuh"
 #include "kernels.h"
+#include "launch_pdl.h"
 
 namespace marche {
 
@@ -27,6 +28,7 @@ attention_simt_kernel(const T* __restrict__ q, int ld_q, int n, int S, int H, in
   extern __shared__ float smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.x / H, h = blockIdx.x % H;
+  pdl_sync();
   const int D = H * dh;
   float* p = smem + (size_t)warp * S;                               // probabilities of the current query
   float* colsum = smem + (size_t)kAttWarps * S + (size_t)warp * S;  // this warp's column sums
@@ -93,15 +95,14 @@ cudaError_t launch_attention_simt(bool bf16_t, const void* q, int ld_q, int B, i
   if (bf16_t) {
     e = cudaFuncSetAttribute(attention_simt_kernel<bf16, f16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attention_simt_kernel<bf16, f16><<<B * H, kAttWarps * 32, smem, st>>>(
-        (const bf16*)q, ld_q, n, S, H, dh, (const bf16*)cache_layer, kv_stride, is_new, score_partial, (f16*)o);
+    return launch_pdl(attention_simt_kernel<bf16, f16>, dim3(B * H), dim3(kAttWarps * 32), smem, st, (const bf16*)q, ld_q,
+                      n, S, H, dh, (const bf16*)cache_layer, kv_stride, is_new, score_partial, (f16*)o);
   } else {
     e = cudaFuncSetAttribute(attention_simt_kernel<float, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attention_simt_kernel<float, float><<<B * H, kAttWarps * 32, smem, st>>>(
-        (const float*)q, ld_q, n, S, H, dh, (const float*)cache_layer, kv_stride, is_new, score_partial, (float*)o);
+    return launch_pdl(attention_simt_kernel<float, float>, dim3(B * H), dim3(kAttWarps * 32), smem, st, (const float*)q,
+                      ld_q, n, S, H, dh, (const float*)cache_layer, kv_stride, is_new, score_partial, (float*)o);
   }
-  return cudaGetLastError();
 }
 
 }  // namespace marche

@@ -8,6 +8,7 @@
 // sample is S^2 integer compares, which at these sizes is latency- not bandwidth-bound.
 #include "common.cuh"
 #include "kernels.h"
+#include "launch_pdl.h"
 
 namespace marche {
 
@@ -27,6 +28,7 @@ topk_kernel(const float* __restrict__ partial, int H, float* __restrict__ scores
   extern __shared__ unsigned long long comp[];          // [S] composite keys; 0 = not a candidate
   __shared__ int warp_tot[kTopkThreads / 32];
   const int b = blockIdx.x, tid = threadIdx.x;
+  pdl_sync();
 
   for (int t = tid; t < S; t += kTopkThreads) {
     float s;
@@ -83,9 +85,8 @@ topk_kernel(const float* __restrict__ partial, int H, float* __restrict__ scores
 cudaError_t launch_topk(const float* partial, int H, float* scores, const uint8_t* cand, int B, int S, int k,
                         int32_t* refresh_idx, cudaStream_t st) {
   if (S > 2048) return cudaErrorInvalidValue;
-  topk_kernel<<<B, kTopkThreads, (size_t)S * sizeof(unsigned long long), st>>>(partial, H, scores, cand, S, k,
-                                                                              refresh_idx);
-  return cudaGetLastError();
+  return launch_pdl(topk_kernel, dim3(B), dim3(kTopkThreads), (size_t)S * sizeof(unsigned long long), st, partial, H,
+                    scores, cand, S, k, refresh_idx);
 }
 
 }  // namespace marche

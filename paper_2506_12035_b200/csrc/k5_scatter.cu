@@ -11,6 +11,7 @@
 // All are pure copies / integer work, bound by HBM (rows) or launch latency (indices).
 #include "common.cuh"
 #include "kernels.h"
+#include "launch_pdl.h"
 
 namespace marche {
 
@@ -22,6 +23,7 @@ scatter_kv_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v, long
   const long w = (long)blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (w >= 2 * total_rows) return;
+  pdl_sync();
   const int which = (int)(w & 1);
   const long r = w >> 1;
   const int b = (int)(r / n), j = (int)(r - (long)b * n);
@@ -37,6 +39,7 @@ scatter_rows_kernel(const float4* __restrict__ rows, const int32_t* __restrict__
   const long r = (long)blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (r >= total_rows) return;
+  pdl_sync();
   const int b = (int)(r / n), j = (int)(r - (long)b * n);
   const int t = idx ? idx[r] : j;
   const float4* src = rows + r * row_vecs;
@@ -50,6 +53,7 @@ gather_rows_kernel(const float4* __restrict__ src, const int32_t* __restrict__ i
   const long r = (long)blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (r >= total_rows) return;
+  pdl_sync();
   const int b = (int)(r / n);
   const float4* s = src + ((long)b * S + idx[r]) * row_vecs;
   float4* d = out + r * row_vecs;
@@ -63,6 +67,7 @@ step_flags_kernel(const int32_t* __restrict__ active_idx, int n_active, const in
                   uint8_t* __restrict__ is_new, uint8_t* __restrict__ cand) {
   extern __shared__ uint8_t mark[];
   const int b = blockIdx.x;
+  pdl_sync();
   for (int t = threadIdx.x; t < S; t += blockDim.x) mark[t] = 0;
   __syncthreads();
   for (int i = threadIdx.x; i < n_new; i += blockDim.x) mark[new_idx[(long)b * n_new + i]] = 1;
@@ -81,6 +86,7 @@ __global__ void build_active_kernel(const int32_t* __restrict__ a, int na, const
   const int n = na + nb + nc;
   const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= (long)B * n) return;
+  pdl_sync();
   const int s = (int)(i / n), j = (int)(i - (long)s * n);
   int32_t v;
   if (j < na) v = a[(long)s * na + j];
@@ -96,6 +102,7 @@ validate_kernel(const int32_t* __restrict__ active_idx, int n_active, const int3
   extern __shared__ int cnt[];
   __shared__ int bad;
   const int b = blockIdx.x;
+  pdl_sync();
   if (threadIdx.x == 0) bad = 0;
   for (int t = threadIdx.x; t < 3 * S; t += blockDim.x) cnt[t] = 0;
   __syncthreads();
@@ -129,9 +136,8 @@ cudaError_t launch_scatter_kv(bool bf16_t, const void* k, const void* v, int ld_
   const long rows = (long)B * n;
   if (rows == 0) return cudaSuccess;
   const unsigned grid = (unsigned)((2 * rows + 7) / 8);
-  scatter_kv_kernel<<<grid, 256, 0, st>>>((const uint4*)k, (const uint4*)v, (long)ld_kv * eb / 16, idx, n, S,
-                                         D * eb / 16, rows, (long)B * S * D * eb / 16, (uint4*)cache_layer);
-  return cudaGetLastError();
+  return launch_pdl(scatter_kv_kernel, dim3(grid), dim3(256), 0, st, (const uint4*)k, (const uint4*)v,
+                    (long)ld_kv * eb / 16, idx, n, S, D * eb / 16, rows, (long)B * S * D * eb / 16, (uint4*)cache_layer);
 }
 
 cudaError_t launch_scatter_rows(const float* rows, const int32_t* idx, int B, int n, int S, int D,
@@ -139,9 +145,8 @@ cudaError_t launch_scatter_rows(const float* rows, const int32_t* idx, int B, in
   if (D % 4) return cudaErrorInvalidValue;
   const long total = (long)B * n;
   if (total == 0) return cudaSuccess;
-  scatter_rows_kernel<<<(unsigned)((total + 7) / 8), 256, 0, st>>>((const float4*)rows, idx, n, S, D / 4, total,
-                                                                  (float4*)dst);
-  return cudaGetLastError();
+  return launch_pdl(scatter_rows_kernel, dim3((unsigned)((total + 7) / 8)), dim3(256), 0, st, (const float4*)rows, idx,
+                    n, S, D / 4, total, (float4*)dst);
 }
 
 cudaError_t launch_gather_rows(const float* src, const int32_t* idx, int B, int n, int S, int D, float* out,
@@ -149,31 +154,29 @@ cudaError_t launch_gather_rows(const float* src, const int32_t* idx, int B, int 
   if (D % 4) return cudaErrorInvalidValue;
   const long total = (long)B * n;
   if (total == 0) return cudaSuccess;
-  gather_rows_kernel<<<(unsigned)((total + 7) / 8), 256, 0, st>>>((const float4*)src, idx, n, S, D / 4, total,
-                                                                 (float4*)out);
-  return cudaGetLastError();
+  return launch_pdl(gather_rows_kernel, dim3((unsigned)((total + 7) / 8)), dim3(256), 0, st, (const float4*)src, idx, n,
+                    S, D / 4, total, (float4*)out);
 }
 
 cudaError_t launch_step_flags(const int32_t* active_idx, int n_active, const int32_t* new_idx, int n_new,
                               const int32_t* excl_idx, int n_excl, int B, int S, uint8_t* is_new,
                               uint8_t* cand, cudaStream_t st) {
-  step_flags_kernel<<<B, 256, S, st>>>(active_idx, n_active, new_idx, n_new, excl_idx, n_excl, S, is_new, cand);
-  return cudaGetLastError();
+  return launch_pdl(step_flags_kernel, dim3(B), dim3(256), (size_t)S, st, active_idx, n_active, new_idx, n_new, excl_idx,
+                    n_excl, S, is_new, cand);
 }
 
 cudaError_t launch_build_active(const int32_t* a, int na, const int32_t* b, int nb, const int32_t* c, int nc,
                                 int B, int32_t* out, cudaStream_t st) {
   const long total = (long)B * (na + nb + nc);
   if (total == 0) return cudaSuccess;
-  build_active_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(a, na, b, nb, c, nc, B, out);
-  return cudaGetLastError();
+  return launch_pdl(build_active_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st, a, na, b, nb, c, nc,
+                    B, out);
 }
 
 cudaError_t launch_validate(const int32_t* active_idx, int n_active, const int32_t* new_idx, int n_new,
                             const int32_t* excl_idx, int n_excl, int B, int S, int* status, cudaStream_t st) {
-  validate_kernel<<<B, 256, 3 * S * sizeof(int), st>>>(active_idx, n_active, new_idx, n_new, excl_idx, n_excl, S,
-                                                      status);
-  return cudaGetLastError();
+  return launch_pdl(validate_kernel, dim3(B), dim3(256), 3 * S * sizeof(int), st, active_idx, n_active, new_idx, n_new,
+                    excl_idx, n_excl, S, status);
 }
 
 }  // namespace marche
