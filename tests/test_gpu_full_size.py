@@ -1,5 +1,6 @@
-"""Parity at the benchmark's full size, in the launch configuration bench.py times: the
-MAR-L-shaped stack (32 blocks, width 1024, 16 heads, S 320) at batch 128.  The GPU runs the
+"""Parity at the full sizes of the benchmark configurations, in the launch configuration
+bench.py times: the MAR-L-shaped stack (32 blocks, width 1024, 16 heads, S 320, batch 128) and
+likewise MAR-B, MAR-H (head_dim 80) and the high-resolution case (S 1088, batch 64).  The GPU runs the
 whole batch; the oracle runs one classifier-free-guidance pair (rows 0 and 64) - samples are
 independent (pinned by the oracle's sample-independence test), so their rows must match the
 oracle's.  One full step and two cache-aware steps, teacher-forced with the oracle's refresh
@@ -15,7 +16,7 @@ from helpers import TOL, dev, idx_dev, make_model, max_abs, rel_l2
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name", ["mar_l"])
+@pytest.mark.parametrize("name", ["mar_l", "mar_b", "mar_h", "hires"])
 def test_full_size_sampled_parity(name):
     cfg = synth.CONFIGS[name]
     if torch.cuda.get_device_properties(0).total_memory < 40e9:
