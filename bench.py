@@ -40,7 +40,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM traffic per launch of the dominant kernel classes from the committed ncu captures
 # (profiles/), bytes; None where no capture exists.
-NCU_TRAFFIC = {"gemm": None, "attention": None}
+NCU_TRAFFIC = {"gemm": 31.1e6,        # profiles/gemm_tcgen05_2cta_mar_l_rows4352.md (mean of the block's four GEMMs)
+               "attention": 183.6e6}  # profiles/attention_mma_mar_l_nA34.md
 
 
 def load_peaks():
@@ -118,7 +119,10 @@ def schedule(cfg, ratio):
 
 
 def algorithmic_work(cfg, sched):
-    """Algorithmic flops / bytes per generation for each kernel class (bf16 operands, fp32 residual)."""
+    """Algorithmic flops / bytes for each kernel class over the given steps (16-bit operands, fp32
+    residual): per step and block, K1 reads M*D*4 and writes M*D*2 (twice per block, plus the compact
+    fp32 copy at block 0); K2 does 2*M*(4*D*D + 2*D*F) flops; K5 moves 2*M*D*2 bytes in and out; K3 reads
+    K and V of all S tokens plus Q and writes O; K4 reads the score partials and the mask."""
     B, S, D, F, L, H = cfg.B, cfg.S, cfg.D, cfg.F, cfg.L, cfg.H
     w = {"gemm_flops": 0.0, "attention_bytes": 0.0, "attention_flops": 0.0, "gather_layernorm_bytes": 0.0,
          "scatter_kv_bytes": 0.0, "scatter_rows_bytes": 0.0, "topk_bytes": 0.0}
@@ -129,9 +133,39 @@ def algorithmic_work(cfg, sched):
         w["attention_flops"] += 4.0 * B * nA * S * D * L
         w["gather_layernorm_bytes"] += 2 * (M * D * 4 + M * D * 2) * L + M * D * 4
         w["scatter_kv_bytes"] += 4.0 * M * D * 2 * L
-        w["scatter_rows_bytes"] += 2.0 * M * D * 4
+        w["scatter_rows_bytes"] += 2.0 * M * D * 4 + 2.0 * B * g * D * 4
         w["topk_bytes"] += B * H * S * 4 + B * S * 5 + B * k * 4
     return w
+
+
+GEMM_CLASSES = ("gemm_qkv", "gemm_out_proj", "gemm_fc1_gelu", "gemm_fc2")
+
+
+def kernel_table(prof, work, peaks, attention_bound):
+    """Per-kernel-class roofline rows from one profile (class -> (ms, launches)) and the
+    algorithmic work of the same steps."""
+    total_ms = sum(v[0] for v in prof.values())
+    rows = []
+
+    def add(name, bound, amount, ms, n, peak, unit):
+        if n == 0 or ms <= 0:
+            return
+        ach = amount / (ms * 1e-3) / (1e12 if unit == "TFLOP/s" else 1e9)
+        rows.append({"kernel": name, "bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                     "launches": n, "ms": ms, "us_per_launch": 1e3 * ms / n, "share": ms / total_ms})
+
+    add("gemm_tcgen05 (qkv, out, fc1, fc2)", "tensor", work["gemm_flops"], sum(prof[c][0] for c in GEMM_CLASSES),
+        sum(prof[c][1] for c in GEMM_CLASSES), peaks["bf16_tflops_sustained"], "TFLOP/s")
+    if attention_bound == "hbm":
+        add("attention", "hbm", work["attention_bytes"], *prof["attention"], peaks["hbm_gbs"], "GB/s")
+    else:
+        add("attention", "tensor", work["attention_flops"], *prof["attention"], peaks["bf16_tflops_sustained"], "TFLOP/s")
+    add("gather_layernorm", "hbm", work["gather_layernorm_bytes"], *prof["gather_layernorm"], peaks["hbm_gbs"], "GB/s")
+    add("scatter_kv", "hbm", work["scatter_kv_bytes"], *prof["scatter_kv"], peaks["hbm_gbs"], "GB/s")
+    add("scatter_rows", "hbm", work["scatter_rows_bytes"], *prof["scatter_rows"], peaks["hbm_gbs"], "GB/s")
+    add("topk", "hbm", work["topk_bytes"], *prof["topk"], peaks["hbm_gbs"], "GB/s")
+    rows.sort(key=lambda r: -r["ms"])
+    return rows
 
 
 # ----------------------------------------------------------------------------- reference arm (CPU oracle)
@@ -270,39 +304,30 @@ def run_ours(args, cfg):
             "ms_per_decoding_step": ms_gen / cfg.T}
 
     if not args.no_extras:
-        # ---- per-kernel-class device time of one more generation (events in front of every launch)
+        # ---- per-kernel-class device time of one more generation (an event in front of every
+        # launch; events serialise the launches, so programmatic dependent launch does not overlap
+        # here and the figures are conservative).  The first (full) step and the cache-aware steps
+        # are accounted separately: the cache-aware step is the hot path proper.
+        profs = {}
+
+        def split(t):
+            if t == 0:
+                profs["full"] = m.profile_end()
+                m.profile_begin()
+
         m.profile_begin()
-        gen.run(hidden0)
-        prof = m.profile_end()
-        gemm_ms = sum(prof[c][0] for c in ("gemm_qkv", "gemm_out_proj", "gemm_fc1_gelu", "gemm_fc2"))
-        gemm_n = sum(prof[c][1] for c in ("gemm_qkv", "gemm_out_proj", "gemm_fc1_gelu", "gemm_fc2"))
-        total_ms = sum(v[0] for v in prof.values())
-        kernels = []
-
-        def add(name, bound, amount, ms, n, peak, unit):
-            if n == 0 or ms <= 0:
-                return
-            ach = amount / (ms * 1e-3) / (1e12 if unit == "TFLOP/s" else 1e9)
-            kernels.append({"kernel": name, "bound": bound, "achieved": ach, "peak": peak, "unit": unit,
-                            "frac": ach / peak, "launches": n, "ms_per_generation": ms, "share": ms / total_ms})
-
-        add("gemm_tcgen05 (qkv, out, fc1, fc2)", "tensor", work["gemm_flops"], gemm_ms, gemm_n,
-            peaks["bf16_tflops_sustained"], "TFLOP/s")
-        add("attention", "hbm", work["attention_bytes"], prof["attention"][0], prof["attention"][1], peaks["hbm_gbs"], "GB/s")
-        add("gather_layernorm", "hbm", work["gather_layernorm_bytes"], prof["gather_layernorm"][0],
-            prof["gather_layernorm"][1], peaks["hbm_gbs"], "GB/s")
-        add("scatter_kv", "hbm", work["scatter_kv_bytes"], prof["scatter_kv"][0], prof["scatter_kv"][1], peaks["hbm_gbs"], "GB/s")
-        add("scatter_rows", "hbm", work["scatter_rows_bytes"], prof["scatter_rows"][0], prof["scatter_rows"][1],
-            peaks["hbm_gbs"], "GB/s")
-        add("topk", "hbm", work["topk_bytes"], prof["topk"][0], prof["topk"][1], peaks["hbm_gbs"], "GB/s")
-        kernels.sort(key=lambda k: -k["ms_per_generation"])
+        gen.run(hidden0, after_step=split)
+        profs["cache_aware"] = m.profile_end()
+        kernels = kernel_table(profs["cache_aware"], algorithmic_work(cfg, sched[1:]), peaks, "hbm")
         line["kernels"] = kernels
+        line["kernels_scope"] = "the %d cache-aware steps of one generation" % (cfg.T - 1)
+        line["full_step_kernels"] = kernel_table(profs["full"], algorithmic_work(cfg, sched[:1]), peaks, "tensor")
         dom = kernels[0]
         key = "gemm" if dom["bound"] == "tensor" else dom["kernel"]
         line["roofline"] = {"kernel": dom["kernel"], "bound": dom["bound"], "achieved": dom["achieved"], "peak": dom["peak"],
                             "unit": dom["unit"], "frac": dom["frac"], "traffic": NCU_TRAFFIC.get(key),
                             "peak_source": "%s (%s)" % (peak_kind, "sustained bf16 GEMM" if dom["bound"] == "tensor" else "device copy"),
-                            "timing": "CUDA events in front of every launch of one generation of the timed workload"}
+                            "timing": "CUDA events in front of every launch, cache-aware steps of one generation of the timed workload"}
 
         # ---- this build's own full-recompute path (full step at every decoding step)
         gen.run(hidden0, mode="full")

@@ -36,7 +36,8 @@ class Generation:
         self.scores = torch.empty(B, S, dtype=torch.float32, device=dev)
 
     def run(self, hidden0: torch.Tensor, mode: str = "marche", record: bool = False,
-            forced_refresh: Optional[List[torch.Tensor]] = None, stream=None, n_steps: Optional[int] = None):
+            forced_refresh: Optional[List[torch.Tensor]] = None, stream=None, n_steps: Optional[int] = None,
+            after_step=None):
         """Enqueues all T steps.  mode "full" runs the full-recompute baseline.  With
         record=True returns per-step host copies (this synchronises every step)."""
         m, B = self.m, self.m.B
@@ -74,6 +75,8 @@ class Generation:
                     hidden_out=self.hidden_out.cpu().numpy().copy()))
             m.scatter_rows(self.rows[t], G, self.hidden, stream)
             k_prev = k
+            if after_step is not None:
+                after_step(t)
         return log
 
     # ------------------------------------------------------------------ host-driven loop
