@@ -180,6 +180,26 @@ int marche_full_step(marche_ctx* ctx, const float* hidden, void* kv_cache,
                      int32_t* refresh_idx, int* n_refresh,
                      void* workspace, size_t workspace_bytes, marche_stream stream);
 
+/* One decoding step under the paper's own schedule (Section 4.2 and Figure 3, Section 4.3):
+ * blocks 0 .. score_layer run full attention on every token (their cache layers are fully
+ * refreshed), the relevance scores are taken at block score_layer from the queries of new_idx,
+ * the n_refresh highest-scoring tokens outside new_idx u prev_idx become the refreshing tokens,
+ * and the blocks after score_layer run cache-aware on A = new | prev | refresh (Algorithm 1).
+ * With a fixed active budget the caller passes n_refresh = budget - n_new - n_prev.
+ *   prev_idx        device int32 [B][n_prev]: tokens generated in the previous step (N), or NULL
+ *   forced_refresh  device int32 [B][n_refresh] or NULL: when given it is used as R instead of the
+ *                   selection (which is still written to refresh_idx) - for teacher-forced tests
+ *   refresh_idx     out, device int32 [B][n_refresh];  active_idx out, device int32 [B][nA],
+ *                   nA = n_new + n_prev + n_refresh
+ *   hidden_out      rows active_idx receive the stack output; other rows keep their bytes
+ *   workspace       marche_workspace_bytes(ctx, S)
+ * Needs score_layer < L-1 (MARCHE_EINVAL otherwise) and a filled cache (MARCHE_ECACHE). */
+int marche_step_in_step_selection(marche_ctx* ctx, const float* hidden, void* kv_cache,
+                                  const int32_t* new_idx, int n_new, const int32_t* prev_idx, int n_prev,
+                                  int n_refresh, const int32_t* forced_refresh, float* hidden_out,
+                                  int32_t* refresh_idx, int32_t* active_idx,
+                                  void* workspace, size_t workspace_bytes, marche_stream stream);
+
 /* Top-K refresh selection alone (Section 4.2, "select the top-K tokens with the
  * highest relevance scores"): scores device float [B][S] (finite); candidates
  * are all tokens outside new_idx and exclude_idx; writes refresh_idx device

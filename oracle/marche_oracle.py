@@ -34,6 +34,10 @@ What is written out, and from where in the paper:
                            full refresh of Section 4.3 and the full-recompute
                            MAR baseline of Section 3 (Motivation).
 * `active_set`             Algorithm 1 line 4: A = G u R u N.
+* `in_step_selection_step` the paper's own schedule of one step (Section 4.2, Figure 3): full
+                           attention up to the scoring block, selection there, cache-aware
+                           blocks after it; `generate_in_step` adds the fixed active budget
+                           and the periodic full refresh of Section 4.3.
 
 Readings where the paper is silent (block internals, tie rule, refresh ratio)
 are listed in the repository's design notes; each is marked "reading" below.
@@ -267,6 +271,85 @@ def full_step(blocks, hidden, cache: KVCache, new_idx, exclude_idx, refresh_rati
                       require_filled=False)
     cache.filled = True
     return out
+
+
+def in_step_selection_step(blocks: Sequence[Block], hidden: np.ndarray, cache: KVCache, new_idx: np.ndarray,
+                           prev_idx: Optional[np.ndarray], n_refresh: int, hidden_out: np.ndarray, *,
+                           n_heads: int, score_layer: int, ln_eps: float = 1e-6, real=np.float64,
+                           forced_refresh: Optional[np.ndarray] = None):
+    """One decoding step under the paper's own schedule (Section 4.2, Figure 3; Section 4.3):
+
+    blocks 0 .. score_layer run full attention on every token ("the active tokens are not yet
+    finalized"), the relevance scores are taken from the generating tokens' queries at block
+    score_layer, the n_refresh highest-scoring tokens outside G u N become the refreshing tokens R,
+    and the blocks after score_layer run cache-aware attention on A = G u N u R.
+    new_idx = G [B][nG], prev_idx = N [B][nN] (the tokens generated in the previous step) or None.
+    `forced_refresh` [B][n_refresh], when given, is used as R instead of the selection (the
+    selection is still returned).  Rows A of hidden_out receive the stack output.
+    Returns (scores fp32 [B][S], refresh_idx int32 [B][n_refresh], active_idx int32 [B][nA])."""
+    if not cache.filled:
+        raise RuntimeError("step before any full step")
+    B, S, D = hidden.shape
+    L = len(blocks)
+    if not (0 <= score_layer < L - 1):
+        raise ValueError("score_layer must leave at least one cache-aware block")
+    blocks = [{k: np.asarray(v, dtype=real) for k, v in blk.items()} for blk in blocks]
+    all_idx = np.arange(S, dtype=np.int64)
+    scores = np.zeros((B, S), dtype=real)
+    X_full = []
+    for b in range(B):
+        new = set(np.asarray(new_idx[b]).tolist())
+        scoring_rows = np.array([t in new for t in range(S)], dtype=bool)
+        X = hidden[b].astype(real)
+        for l in range(score_layer + 1):
+            X, sc = _block(X, blocks[l], cache.K[l, b], cache.V[l, b], all_idx, n_heads, ln_eps,
+                           scoring_rows if l == score_layer else None)
+            if sc is not None:
+                scores[b] = sc
+        X_full.append(X)
+    scores32 = scores.astype(np.float32)
+    refresh = select_refresh(scores32, new_idx, prev_idx, n_refresh)
+    R = refresh if forced_refresh is None else np.asarray(forced_refresh, dtype=np.int32)
+    A = active_set(new_idx, prev_idx, R)
+    for b in range(B):
+        idx = A[b].astype(np.int64)
+        X = X_full[b][idx]
+        for l in range(score_layer + 1, L):
+            X, _ = _block(X, blocks[l], cache.K[l, b], cache.V[l, b], idx, n_heads, ln_eps, None)
+        hidden_out[b, idx] = X.astype(hidden_out.dtype)
+    return scores32, refresh, A
+
+
+def generate_in_step(blocks, hidden0: np.ndarray, new_sets: List[np.ndarray], replacement, *, n_heads: int,
+                     score_layer: int, budget: int = 64, period: int = 3, ln_eps: float = 1e-6, real=np.float64):
+    """The paper's schedule over a whole generation (Section 4.3): the first step and every
+    `period`-th step refresh the whole cache with a full step; the others use
+    in_step_selection_step with a fixed active budget, K = budget - #G - #N (clipped to the
+    number of candidates).  Returns per-step dicts and the final cache."""
+    B, S, D = hidden0.shape
+    hidden = hidden0.copy()
+    hidden_out = np.zeros_like(hidden0)
+    cache = KVCache(len(blocks), B, S, D, real=real)
+    empty = np.zeros((B, 0), dtype=np.int32)
+    log = []
+    kw = dict(n_heads=n_heads, score_layer=score_layer, ln_eps=ln_eps, real=real)
+    for t, G in enumerate(new_sets):
+        N = new_sets[t - 1] if t > 0 else empty
+        if t % period == 0:
+            A = np.tile(np.arange(S, dtype=np.int32), (B, 1))
+            scores, _ = full_step(blocks, hidden, cache, G, None, 0.0, hidden_out, **kw)
+            R = empty
+            kind = "full"
+        else:
+            k = min(fixed_budget_refresh_count(budget, G.shape[1], N.shape[1]), S - G.shape[1] - N.shape[1])
+            scores, R, A = in_step_selection_step(blocks, hidden, cache, G, N, k, hidden_out, **kw)
+            kind = "in_step"
+        log.append(dict(t=t, kind=kind, active=A, new=G, prev=N, scores=scores, refresh=R,
+                        hidden_out=hidden_out.copy()))
+        rows = replacement(t, G.shape[1])
+        for b in range(B):
+            hidden[b, G[b]] = rows[b]
+    return log, cache
 
 
 # --------------------------------------------------------------------------

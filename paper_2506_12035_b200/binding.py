@@ -49,6 +49,7 @@ _SIGNATURES = {
     "marche_init_cache": (C.c_int, [_vp, _vp, _sz, _vp]),
     "marche_step": (C.c_int, [_vp, _vp, _vp, _vp, _i, _vp, _i, _vp, _i, _f, _vp, _vp, C.POINTER(C.c_int), _vp, _sz, _vp]),
     "marche_full_step": (C.c_int, [_vp, _vp, _vp, _vp, _i, _vp, _i, _f, _vp, _vp, C.POINTER(C.c_int), _vp, _sz, _vp]),
+    "marche_step_in_step_selection": (C.c_int, [_vp, _vp, _vp, _vp, _i, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "marche_select_refresh": (C.c_int, [_vp, _vp, _vp, _i, _vp, _i, _i, _vp, _vp, _vp]),
     "marche_select_refresh_static": (C.c_int, [_vp, _vp, _vp, _i, _vp, _i, _i, _vp, _vp]),
     "marche_get_scores": (C.c_int, [_vp, _vp, _vp, _vp]),
@@ -206,6 +207,13 @@ class Marche:
             refresh_ratio, _ptr(hidden_out), _ptr(refresh_idx), C.byref(k), _ptr(workspace), workspace.numel(),
             _stream(stream)))
         return k.value
+
+    def step_in_step_selection(self, hidden, kv_cache, new_idx, prev_idx, n_refresh, forced_refresh, hidden_out,
+                               refresh_idx, active_idx, workspace, stream=None):
+        self._check(self.lib.marche_step_in_step_selection(
+            self.h, _ptr(hidden), _ptr(kv_cache), _ptr(new_idx), 0 if new_idx is None else new_idx.shape[1],
+            _ptr(prev_idx), 0 if prev_idx is None else prev_idx.shape[1], n_refresh, _ptr(forced_refresh),
+            _ptr(hidden_out), _ptr(refresh_idx), _ptr(active_idx), _ptr(workspace), workspace.numel(), _stream(stream)))
 
     def select_refresh(self, scores, new_idx, exclude_idx, k, refresh_idx, mask_scratch, stream=None):
         self._check(self.lib.marche_select_refresh(

@@ -50,7 +50,7 @@ namespace {
 inline size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 struct WsLayout {
-  size_t scores, partial, cand, is_new, x, u, qkv, o, g, total;
+  size_t scores, partial, cand, is_new, x, x2, u, qkv, o, g, total;
 };
 
 WsLayout ws_layout(const marche_ctx* c, int nA) {
@@ -63,6 +63,7 @@ WsLayout ws_layout(const marche_ctx* c, int nA) {
   w.cand = off;    off += align256(B * S);
   w.is_new = off;  off += align256(M);
   w.x = off;       off += align256(M * D * sizeof(float));
+  w.x2 = off;      off += align256(M * D * sizeof(float));   // second residual buffer (in-step selection)
   w.u = off;       off += align256(M * D * eb);
   w.qkv = off;     off += align256(M * 3 * D * eb);
   w.o = off;       off += align256(M * D * eb);
@@ -132,13 +133,75 @@ int do_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void* ca
   return MARCHE_OK;
 }
 
+struct StackBufs {
+  float* scores; float* partial; uint8_t* cand; uint8_t* is_new;
+  float* x; float* x2; char* u; char* qkv; char* o; char* g;
+};
+
+StackBufs carve(void* workspace, const WsLayout& w) {
+  char* ws = (char*)workspace;
+  StackBufs b;
+  b.scores = (float*)(ws + w.scores);
+  b.partial = (float*)(ws + w.partial);
+  b.cand = (uint8_t*)(ws + w.cand);
+  b.is_new = (uint8_t*)(ws + w.is_new);
+  b.x = (float*)(ws + w.x);
+  b.x2 = (float*)(ws + w.x2);
+  b.u = ws + w.u;
+  b.qkv = ws + w.qkv;
+  b.o = ws + w.o;
+  b.g = ws + w.g;
+  return b;
+}
+
+// Blocks [l_begin, l_end) for M = B*nA rows whose token positions are idx (nullptr = identity,
+// nA == S).  When gather_src is non-null the first block's LayerNorm gathers its rows from
+// gather_src[b][idx][:] (float [B][src_rows][D]) and writes the compact residual rows to x;
+// otherwise x already holds them.  is_new (flags of the scoring queries) is used at the scoring block.
+int run_blocks(marche_ctx* ctx, int l_begin, int l_end, const float* gather_src, int src_rows, const int32_t* idx,
+               int nA, float* x, const StackBufs& bf, void* kv_cache, const uint8_t* is_new, cudaStream_t st) {
+  const marche_config& c = ctx->cfg;
+  const int B = c.batch, S = c.seq_len, D = c.width, F = c.mlp_dim;
+  const int M = B * nA;
+  const size_t eb = ctx->eb;
+  const size_t layer_bytes = (size_t)2 * B * S * D * eb;
+  for (int l = l_begin; l < l_end; ++l) {
+    const marche_block_weights& bw = ctx->blocks[l];
+    char* cache_l = (char*)kv_cache + (size_t)l * layer_bytes;
+    mark(ctx, MARCHE_KC_GATHER_LN, st);
+    if (l == l_begin && gather_src)
+      MARCHE_TRY(launch_gather_layernorm(ctx->bf16, gather_src, src_rows, idx, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
+                                         x, bf.u, st), "gather_layernorm");
+    else
+      MARCHE_TRY(launch_gather_layernorm(ctx->bf16, x, nA, nullptr, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
+                                         nullptr, bf.u, st), "layernorm1");
+    int rc = do_linear(ctx, MARCHE_KC_GEMM_QKV, bf.u, D, M, bw.w_qkv, bw.b_qkv, 3 * D, D, MARCHE_EPI_BIAS, bf.qkv, st);
+    if (rc) return rc;
+    mark(ctx, MARCHE_KC_SCATTER_KV, st);
+    MARCHE_TRY(launch_scatter_kv(ctx->bf16, bf.qkv + (size_t)D * eb, bf.qkv + (size_t)2 * D * eb, 3 * D, idx, B, nA,
+                                 S, D, cache_l, st), "scatter_kv");
+    rc = do_attention(ctx, bf.qkv, 3 * D, nA, cache_l, l == ctx->score_layer ? is_new : nullptr, bf.partial, bf.o, st);
+    if (rc) return rc;
+    rc = do_linear(ctx, MARCHE_KC_GEMM_O, bf.o, D, M, bw.w_o, bw.b_o, D, D, MARCHE_EPI_BIAS_RESIDUAL, x, st);
+    if (rc) return rc;
+    mark(ctx, MARCHE_KC_GATHER_LN, st);
+    MARCHE_TRY(launch_gather_layernorm(ctx->bf16, x, nA, nullptr, B, nA, D, bw.ln2_g, bw.ln2_b, ctx->eps, nullptr,
+                                       bf.u, st), "layernorm2");
+    rc = do_linear(ctx, MARCHE_KC_GEMM_FC1, bf.u, D, M, bw.w_fc1, bw.b_fc1, F, D, MARCHE_EPI_BIAS_GELU, bf.g, st);
+    if (rc) return rc;
+    rc = do_linear(ctx, MARCHE_KC_GEMM_FC2, bf.g, F, M, bw.w_fc2, bw.b_fc2, D, F, MARCHE_EPI_BIAS_RESIDUAL, x, st);
+    if (rc) return rc;
+  }
+  return MARCHE_OK;
+}
+
 // The whole stack for M = B*nA rows.  active_idx == nullptr means every token (nA == S).
 int run_stack(marche_ctx* ctx, const float* hidden, void* kv_cache, const int32_t* active_idx, int nA,
               const int32_t* new_idx, int n_new, const int32_t* excl_idx, int n_excl, float ratio,
               float* hidden_out, int32_t* refresh_idx, int* n_refresh, void* workspace, size_t ws_bytes,
               cudaStream_t st) {
   const marche_config& c = ctx->cfg;
-  const int B = c.batch, S = c.seq_len, D = c.width, F = c.mlp_dim, H = c.n_heads, L = c.n_blocks;
+  const int B = c.batch, S = c.seq_len, D = c.width, H = c.n_heads, L = c.n_blocks;
   if (!hidden || !kv_cache || !hidden_out || !workspace || hidden == hidden_out) return MARCHE_EINVAL;
   if (nA < 1 || nA > S || n_new < 0 || n_new > nA || n_excl < 0 || n_new + n_excl > S) return MARCHE_EINVAL;
   if ((n_new > 0 && !new_idx) || (n_excl > 0 && !excl_idx)) return MARCHE_EINVAL;
@@ -147,54 +210,52 @@ int run_stack(marche_ctx* ctx, const float* hidden, void* kv_cache, const int32_
   if (ws_bytes < w.total) return MARCHE_EWORKSPACE;
   const int k = refresh_idx ? refresh_count(ratio, S, S - n_new - n_excl) : 0;
   if (n_refresh) *n_refresh = k;
-
-  char* ws = (char*)workspace;
-  float* scores = (float*)(ws + w.scores);
-  float* partial = (float*)(ws + w.partial);
-  uint8_t* cand = (uint8_t*)(ws + w.cand);
-  uint8_t* is_new = (uint8_t*)(ws + w.is_new);
-  float* x = (float*)(ws + w.x);
-  char* u = ws + w.u;
-  char* qkv = ws + w.qkv;
-  char* o = ws + w.o;
-  char* g = ws + w.g;
-  const int M = B * nA;
-  const size_t eb = ctx->eb;
-  const size_t layer_bytes = (size_t)2 * B * S * D * eb;
+  const StackBufs bf = carve(workspace, w);
 
   mark(ctx, MARCHE_KC_FLAGS, st);
-  MARCHE_TRY(launch_step_flags(active_idx, nA, new_idx, n_new, excl_idx, n_excl, B, S, is_new, cand, st), "flags");
-  for (int l = 0; l < L; ++l) {
-    const marche_block_weights& bw = ctx->blocks[l];
-    char* cache_l = (char*)kv_cache + (size_t)l * layer_bytes;
-    mark(ctx, MARCHE_KC_GATHER_LN, st);
-    if (l == 0)
-      MARCHE_TRY(launch_gather_layernorm(ctx->bf16, hidden, S, active_idx, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
-                                         x, u, st), "gather_layernorm");
-    else
-      MARCHE_TRY(launch_gather_layernorm(ctx->bf16, x, nA, nullptr, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
-                                         nullptr, u, st), "layernorm1");
-    int rc = do_linear(ctx, MARCHE_KC_GEMM_QKV, u, D, M, bw.w_qkv, bw.b_qkv, 3 * D, D, MARCHE_EPI_BIAS, qkv, st);
-    if (rc) return rc;
-    mark(ctx, MARCHE_KC_SCATTER_KV, st);
-    MARCHE_TRY(launch_scatter_kv(ctx->bf16, qkv + (size_t)D * eb, qkv + (size_t)2 * D * eb, 3 * D, active_idx, B, nA,
-                                 S, D, cache_l, st), "scatter_kv");
-    rc = do_attention(ctx, qkv, 3 * D, nA, cache_l, l == ctx->score_layer ? is_new : nullptr, partial, o, st);
-    if (rc) return rc;
-    rc = do_linear(ctx, MARCHE_KC_GEMM_O, o, D, M, bw.w_o, bw.b_o, D, D, MARCHE_EPI_BIAS_RESIDUAL, x, st);
-    if (rc) return rc;
-    mark(ctx, MARCHE_KC_GATHER_LN, st);
-    MARCHE_TRY(launch_gather_layernorm(ctx->bf16, x, nA, nullptr, B, nA, D, bw.ln2_g, bw.ln2_b, ctx->eps, nullptr,
-                                       u, st), "layernorm2");
-    rc = do_linear(ctx, MARCHE_KC_GEMM_FC1, u, D, M, bw.w_fc1, bw.b_fc1, F, D, MARCHE_EPI_BIAS_GELU, g, st);
-    if (rc) return rc;
-    rc = do_linear(ctx, MARCHE_KC_GEMM_FC2, g, F, M, bw.w_fc2, bw.b_fc2, D, F, MARCHE_EPI_BIAS_RESIDUAL, x, st);
-    if (rc) return rc;
-  }
+  MARCHE_TRY(launch_step_flags(active_idx, nA, new_idx, n_new, excl_idx, n_excl, B, S, bf.is_new, bf.cand, st), "flags");
+  const int rc = run_blocks(ctx, 0, L, hidden, S, active_idx, nA, bf.x, bf, kv_cache, bf.is_new, st);
+  if (rc) return rc;
   mark(ctx, MARCHE_KC_SCATTER_ROWS, st);
-  MARCHE_TRY(launch_scatter_rows(x, active_idx, B, nA, S, D, hidden_out, st), "scatter_rows");
+  MARCHE_TRY(launch_scatter_rows(bf.x, active_idx, B, nA, S, D, hidden_out, st), "scatter_rows");
   mark(ctx, MARCHE_KC_TOPK, st);
-  MARCHE_TRY(launch_topk(partial, H, scores, cand, B, S, k, refresh_idx, st), "topk");
+  MARCHE_TRY(launch_topk(bf.partial, H, bf.scores, bf.cand, B, S, k, refresh_idx, st), "topk");
+  return MARCHE_OK;
+}
+
+// One step under the paper's own schedule: blocks 0..score_layer on every token, top-K there,
+// blocks after it on A = new | prev | refresh.
+int run_in_step(marche_ctx* ctx, const float* hidden, void* kv_cache, const int32_t* new_idx, int n_new,
+                const int32_t* prev_idx, int n_prev, int k, const int32_t* forced_refresh, float* hidden_out,
+                int32_t* refresh_idx, int32_t* active_idx, void* workspace, size_t ws_bytes, cudaStream_t st) {
+  const marche_config& c = ctx->cfg;
+  const int B = c.batch, S = c.seq_len, D = c.width, H = c.n_heads, L = c.n_blocks, sl = ctx->score_layer;
+  if (!hidden || !kv_cache || !hidden_out || !workspace || !refresh_idx || !active_idx || hidden == hidden_out)
+    return MARCHE_EINVAL;
+  if (n_new < 0 || n_prev < 0 || k < 0 || n_new + n_prev + k > S || n_new + n_prev + k < 1) return MARCHE_EINVAL;
+  if ((n_new > 0 && !new_idx) || (n_prev > 0 && !prev_idx)) return MARCHE_EINVAL;
+  if (sl >= L - 1) return MARCHE_EINVAL;                     // needs at least one cache-aware block
+  if (((uintptr_t)workspace & 255) != 0) return MARCHE_EINVAL;
+  const WsLayout w = ws_layout(ctx, S);
+  if (ws_bytes < w.total) return MARCHE_EWORKSPACE;
+  const StackBufs bf = carve(workspace, w);
+  const int nA = n_new + n_prev + k;
+
+  // phase 1: every token; generating rows flagged for the scores; candidates = all \ (new u prev)
+  mark(ctx, MARCHE_KC_FLAGS, st);
+  MARCHE_TRY(launch_step_flags(nullptr, S, new_idx, n_new, prev_idx, n_prev, B, S, bf.is_new, bf.cand, st), "flags");
+  int rc = run_blocks(ctx, 0, sl + 1, hidden, S, nullptr, S, bf.x, bf, kv_cache, bf.is_new, st);
+  if (rc) return rc;
+  mark(ctx, MARCHE_KC_TOPK, st);
+  MARCHE_TRY(launch_topk(bf.partial, H, bf.scores, bf.cand, B, S, k, refresh_idx, st), "topk");
+  mark(ctx, MARCHE_KC_OTHER, st);
+  MARCHE_TRY(launch_build_active(new_idx, n_new, prev_idx, n_prev, forced_refresh ? forced_refresh : refresh_idx, k, B,
+                                 active_idx, st), "build_active");
+  // phase 2: rows of A, gathered from the full residual rows of phase 1
+  rc = run_blocks(ctx, sl + 1, L, bf.x, S, active_idx, nA, bf.x2, bf, kv_cache, nullptr, st);
+  if (rc) return rc;
+  mark(ctx, MARCHE_KC_SCATTER_ROWS, st);
+  MARCHE_TRY(launch_scatter_rows(bf.x2, active_idx, B, nA, S, D, hidden_out, st), "scatter_rows");
   return MARCHE_OK;
 }
 
@@ -300,6 +361,17 @@ int marche_full_step(marche_ctx* ctx, const float* hidden, void* kv_cache, const
     else ctx->caches.emplace_back(kv_cache, true);
   }
   return rc;
+}
+
+int marche_step_in_step_selection(marche_ctx* ctx, const float* hidden, void* kv_cache, const int32_t* new_idx,
+                                  int n_new, const int32_t* prev_idx, int n_prev, int n_refresh,
+                                  const int32_t* forced_refresh, float* hidden_out, int32_t* refresh_idx,
+                                  int32_t* active_idx, void* workspace, size_t workspace_bytes, marche_stream stream) {
+  if (!ctx) return MARCHE_EINVAL;
+  auto* e = find_cache(ctx, kv_cache);
+  if (!e || !e->second) return MARCHE_ECACHE;
+  return run_in_step(ctx, hidden, kv_cache, new_idx, n_new, prev_idx, n_prev, n_refresh, forced_refresh, hidden_out,
+                     refresh_idx, active_idx, workspace, workspace_bytes, (cudaStream_t)stream);
 }
 
 int marche_select_refresh(marche_ctx* ctx, const float* scores, const int32_t* new_idx, int n_new,

@@ -79,6 +79,40 @@ class Generation:
                 after_step(t)
         return log
 
+    # ------------------------------------------------------------------ the paper's own schedule
+    def run_in_step(self, hidden0: torch.Tensor, budget: int = 64, period: int = 3, record: bool = False,
+                    forced_refresh: Optional[List[Optional[torch.Tensor]]] = None, stream=None,
+                    n_steps: Optional[int] = None):
+        """Section 4.3 schedule: a full step at t = 0 and every `period`-th step, otherwise
+        marche_step_in_step_selection with K = budget - #G - #N refreshing tokens."""
+        m, B, S = self.m, self.m.B, self.m.S
+        self.hidden.copy_(hidden0, non_blocking=True)
+        m.init_cache(self.cache, stream)
+        log = []
+        for t in range(self.T if n_steps is None else min(n_steps, self.T)):
+            G = self.new_sets[t]
+            N = self.new_sets[t - 1] if t > 0 else None
+            if t % period == 0:
+                m.full_step(self.hidden, self.cache, G, None, 0.0, self.hidden_out, None, self.workspace, stream)
+                n_active, k, active = S, 0, None
+            else:
+                n_gn = G.shape[1] + N.shape[1]
+                k = min(max(0, budget - n_gn), S - n_gn)
+                n_active = n_gn + k
+                active = self.active_flat[: B * n_active].view(B, n_active)
+                fr = None if forced_refresh is None else forced_refresh[t]
+                m.step_in_step_selection(self.hidden, self.cache, G, N, k, fr, self.hidden_out, self.refresh_flat[0],
+                                         active, self.workspace, stream)
+            if record:
+                m.get_scores(self.workspace, self.scores, stream)
+                torch.cuda.synchronize()
+                log.append(dict(t=t, n_active=n_active, active=None if active is None else active.cpu().numpy().copy(),
+                                scores=self.scores.cpu().numpy().copy(),
+                                refresh=self.refresh_flat[0][: B * k].view(B, k).cpu().numpy().copy(),
+                                hidden_out=self.hidden_out.cpu().numpy().copy()))
+            m.scatter_rows(self.rows[t], G, self.hidden, stream)
+        return log
+
     # ------------------------------------------------------------------ host-driven loop
     def alloc_host_buffers(self, hidden0, rows_np, sets_np):
         """Pinned host buffers for run_host: the stack input, per step the sampled rows and

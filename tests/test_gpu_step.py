@@ -168,6 +168,48 @@ def test_full_ratio_equals_full_recompute():
     assert max_abs(host(cache_m), host(gen.cache)) <= 2e-2
 
 
+@pytest.mark.parametrize("case", ["tiny_f32", "tiny_bf16", "marb_slice"])
+def test_in_step_selection_schedule(case):
+    """The paper's own schedule (full attention up to the scoring block, selection there,
+    cache-aware blocks after it; fixed active budget; periodic full refresh), teacher-forced
+    with the oracle's refresh sets."""
+    cfg = CASES[case]
+    if cfg.score_layer >= cfg.L - 1:
+        cfg = cfg.replace(E=cfg.E - 1)
+    budget = 24 if cfg.S < 100 else 64
+    blocks = synth.make_weights(cfg)
+    hidden0 = synth.make_hidden(cfg)
+    sets = synth.new_token_sets(cfg, synth.generation_orders(cfg))
+    log, cache = orc.generate_in_step(blocks, hidden0, sets, lambda t, n: synth.replacement_rows(cfg, t, n),
+                                      n_heads=cfg.H, score_layer=cfg.score_layer, budget=budget, period=3,
+                                      ln_eps=cfg.ln_eps)
+    m, gen = gpu_generation(cfg, blocks, sets, 0.0)
+    forced = [idx_dev(r["refresh"]) if r["kind"] == "in_step" and r["refresh"].shape[1] else None for r in log]
+    glog = gen.run_in_step(dev(hidden0), budget=budget, period=3, record=True, forced_refresh=forced)
+    assert m.device_status() == 0
+    mask = torch.empty(cfg.B * cfg.S, dtype=torch.uint8, device="cuda")
+    for rec, g in zip(log, glog):
+        A = rec["active"]
+        assert g["n_active"] == A.shape[1]
+        if rec["kind"] == "in_step":
+            assert np.array_equal(g["active"], A)
+            assert A.shape[1] == min(budget, cfg.S) or rec["new"].shape[1] + rec["prev"].shape[1] >= budget
+        for b in range(cfg.B):
+            assert_close(g["hidden_out"][b, A[b]], rec["hidden_out"][b, A[b]], cfg.dtype,
+                         "%s step %d (%s)" % (case, rec["t"], rec["kind"]))
+        nG = rec["new"].shape[1]
+        unit = cfg.H * nG / cfg.S
+        assert max_abs(g["scores"], rec["scores"]) <= (5e-2 if cfg.dtype == "bf16" else 1e-4) * unit
+        k = rec["refresh"].shape[1]
+        if k:   # fed the oracle's scores, the device's selection is bit-exact
+            out = torch.empty(cfg.B, k, dtype=torch.int32, device="cuda")
+            m.select_refresh(dev(rec["scores"]), idx_dev(rec["new"]), idx_dev(rec["prev"]), k, out, mask)
+            assert np.array_equal(out.cpu().numpy(), rec["refresh"])
+    K, V = cache_to_oracle_layout(gen.cache)
+    assert_close(K, cache.K, cfg.dtype, case + " cache K")
+    assert_close(V, cache.V, cfg.dtype, case + " cache V")
+
+
 def test_host_driven_step_matches_device_loop():
     """marche_step_host (inputs and results in host buffers) reproduces the device-resident
     loop bit for bit: same kernels, same order; only the copies differ."""

@@ -332,6 +332,55 @@ def test_P11_order_and_sample_independence():
     assert not np.array_equal(out[1], res[0][0][1])
 
 
+def test_in_step_selection_schedule_pins():
+    """The paper's own schedule (Section 4.2-4.3): with every candidate refreshed it equals a
+    full step (Appendix A); the blocks up to the scoring block always hold a fully fresh cache;
+    only rows of A change beyond it; the fixed budget fixes #A."""
+    cfg = small_cfg(L=4, E=1)                      # score layer 2, blocks 3 cache-aware
+    blocks, hidden = setup(cfg)
+    sl = cfg.score_layer
+    sets = synth.new_token_sets(cfg, synth.generation_orders(cfg))
+    G, N = sets[2], sets[1]
+    cache0, _, _, _ = fresh_full(cfg, blocks, hidden, np.zeros((cfg.B, 0), np.int32))
+    rng = np.random.default_rng(3)
+    h2 = hidden.copy()
+    for b in range(cfg.B):
+        h2[b, N[b]] = rng.standard_normal((N.shape[1], cfg.D))
+    cache_f, out_f, sc_f, _ = fresh_full(cfg, blocks, h2, G)
+    kws = dict(n_heads=cfg.H, score_layer=sl, ln_eps=cfg.ln_eps)
+    # (a) K = every candidate: A = all tokens -> the full step
+    c = cache0.copy()
+    out = np.zeros_like(hidden)
+    k_all = cfg.S - G.shape[1] - N.shape[1]
+    sc, R, A = orc.in_step_selection_step(blocks, h2, c, G, N, k_all, out, **kws)
+    assert A.shape[1] == cfg.S and np.array_equal(sc, sc_f)
+    assert np.allclose(out, out_f, rtol=1e-5, atol=1e-6) and np.allclose(c.K, cache_f.K, rtol=1e-9, atol=1e-11)
+    # (b) small K: blocks <= score layer are exactly the full step's, later blocks change only on A
+    c = cache0.copy()
+    out = np.full_like(hidden, 777.0)
+    sc, R, A = orc.in_step_selection_step(blocks, h2, c, G, N, 3, out, **kws)
+    assert A.shape[1] == G.shape[1] + N.shape[1] + 3 and np.array_equal(sc, sc_f)
+    assert np.array_equal(c.K[: sl + 1], cache_f.K[: sl + 1]) and np.array_equal(c.V[: sl + 1], cache_f.V[: sl + 1])
+    for b in range(cfg.B):
+        rest = np.setdiff1d(np.arange(cfg.S), A[b])
+        assert np.array_equal(c.K[sl + 1:, b, rest], cache0.K[sl + 1:, b, rest])
+        assert (out[b, rest] == 777.0).all() and (out[b, A[b]] != 777.0).all()
+        # the refreshing tokens are the top-3 by score among tokens outside G u N
+        cand = [t for t in range(cfg.S) if t not in set(G[b].tolist()) | set(N[b].tolist())]
+        best = sorted(cand, key=lambda t: (-float(sc[b, t]), t))[:3]
+        assert sorted(best) == R[b].tolist()
+    # (c) forced refresh set is honoured but the selection is still reported
+    c2 = cache0.copy()
+    forced = np.stack([np.array([t for t in range(cfg.S) if t not in set(G[b].tolist()) | set(N[b].tolist())][:3]) for b in range(cfg.B)]).astype(np.int32)
+    sc2, R2, A2 = orc.in_step_selection_step(blocks, h2, c2, G, N, 3, np.zeros_like(hidden), forced_refresh=forced, **kws)
+    assert np.array_equal(R2, R) and np.array_equal(A2[:, -3:], forced)
+    # (d) whole generation: full step at t = 0 and every 3rd step, fixed budget elsewhere
+    log, _ = orc.generate_in_step(blocks, hidden, sets, lambda t, n: synth.replacement_rows(cfg, t, n),
+                                  n_heads=cfg.H, score_layer=sl, budget=12, period=3)
+    assert [r["kind"] for r in log] == ["full", "in_step", "in_step", "full"]
+    assert log[1]["active"].shape[1] == 12 and log[2]["active"].shape[1] == 12
+
+
 def test_float32_variant_agrees():
     cfg = small_cfg()
     blocks, hidden = setup(cfg)
