@@ -334,6 +334,21 @@ int marche_scatter_kv(marche_ctx* ctx, const void* k, const void* v, int ld_kv,
 int marche_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void* cache_layer,
                      const uint8_t* is_new, float* score_partial, void* o, marche_stream stream);
 
+/* The paper's own attention kernel shape (Section 4.1, Appendix A.2 and B): the active queries
+ * attend to the fresh segment (K_A, V_A) and to the cached segment (K_C, V_C) separately, the two
+ * are merged with one shared maximum and normaliser (Eq. 6-10), nothing is concatenated, and the
+ * cache rows of the active tokens are written afterwards (Algorithm 1 line 11) by the same kernel.
+ *   qkv   T [B*n][ld]: columns 0..D-1 hold q, D..2D-1 the fresh k, 2D..3D-1 the fresh v (the QKV
+ *         projection's output, read in place); ld >= 3D, ld % 8 == 0
+ *   active_idx  device int32 [B][n] (token of each row; NULL = identity, n == S)
+ *   cache_layer i/o T [2][B][S][D]: rows outside active_idx are read, rows active_idx are written
+ *   is_new / score_partial / o  as for marche_attention
+ * Results equal marche_scatter_kv followed by marche_attention.  MARCHE_BF16 contexts only
+ * (MARCHE_ESHAPE otherwise).  MARCHE_ATTN=twoseg makes the step use this kernel. */
+int marche_attention_two_segment(marche_ctx* ctx, const void* qkv, int ld, int n, const int32_t* active_idx,
+                                 void* cache_layer, const uint8_t* is_new, float* score_partial, void* o,
+                                 marche_stream stream);
+
 /* ---------------------------------------------------------------- diagnostics */
 const char* marche_strerror(int code);
 /* Text of the last CUDA error this context saw ("" if none). */

@@ -60,6 +60,7 @@ _SIGNATURES = {
     "marche_linear": (C.c_int, [_vp, _vp, _i, _i, _vp, _vp, _i, _i, _i, _vp, _vp]),
     "marche_scatter_kv": (C.c_int, [_vp, _vp, _vp, _i, _vp, _i, _vp, _vp]),
     "marche_attention": (C.c_int, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
+    "marche_attention_two_segment": (C.c_int, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "marche_gather_rows": (C.c_int, [_vp, _vp, _vp, _i, _vp, _vp]),
     "marche_staging_bytes": (_sz, [_vp, _i]),
     "marche_step_host": (C.c_int, [_vp, _i, _vp, _vp, _vp, _vp, _i, _vp, _i, _vp, _i, _vp, _i, _f, _vp, _vp, _vp, _vp,
@@ -269,6 +270,11 @@ class Marche:
     def attention(self, q, ld_q, n, cache_layer, is_new, score_partial, o, stream=None):
         self._check(self.lib.marche_attention(self.h, q.data_ptr(), ld_q, n, _ptr(cache_layer), _ptr(is_new),
                                               _ptr(score_partial), _ptr(o), _stream(stream)))
+
+    def attention_two_segment(self, qkv, ld, n, active_idx, cache_layer, is_new, score_partial, o, stream=None):
+        self._check(self.lib.marche_attention_two_segment(self.h, qkv.data_ptr(), ld, n, _ptr(active_idx),
+                                                          _ptr(cache_layer), _ptr(is_new), _ptr(score_partial), _ptr(o),
+                                                          _stream(stream)))
 
     def gather_rows(self, src, idx, rows_out, stream=None):
         self._check(self.lib.marche_gather_rows(self.h, _ptr(src), _ptr(idx), idx.shape[1], _ptr(rows_out),

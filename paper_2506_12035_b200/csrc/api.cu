@@ -33,6 +33,7 @@ struct marche_ctx {
   float eps = 1e-6f;
   int score_layer = 0;
   bool force_simt = false;
+  int attn_mode = 0;                                  // 0 write-back kernel + one-segment attention, 1 two-segment (MARCHE_ATTN)
   int gemm_mode = 0;                                  // 0 auto, 1 single-CTA MMA, 2 CTA-pair MMA (MARCHE_GEMM)
   std::vector<std::pair<const void*, bool>> caches;  // (cache pointer, filled)
   int* status_host = nullptr;                         // pinned, mapped
@@ -177,11 +178,19 @@ int run_blocks(marche_ctx* ctx, int l_begin, int l_end, const float* gather_src,
                                          nullptr, bf.u, st), "layernorm1");
     int rc = do_linear(ctx, MARCHE_KC_GEMM_QKV, bf.u, D, M, bw.w_qkv, bw.b_qkv, 3 * D, D, MARCHE_EPI_BIAS, bf.qkv, st);
     if (rc) return rc;
-    mark(ctx, MARCHE_KC_SCATTER_KV, st);
-    MARCHE_TRY(launch_scatter_kv(ctx->bf16, bf.qkv + (size_t)D * eb, bf.qkv + (size_t)2 * D * eb, 3 * D, idx, B, nA,
-                                 S, D, cache_l, st), "scatter_kv");
-    rc = do_attention(ctx, bf.qkv, 3 * D, nA, cache_l, l == ctx->score_layer ? is_new : nullptr, bf.partial, bf.o, st);
-    if (rc) return rc;
+    if (ctx->attn_mode == 1 && ctx->bf16 && !ctx->force_simt) {
+      // two-segment attention: fresh K/V read in place, cache write-back by the same kernel
+      mark(ctx, MARCHE_KC_ATTENTION, st);
+      MARCHE_TRY(launch_attention_twoseg(bf.qkv, 3 * D, D, 2 * D, B, nA, S, c.n_heads, c.head_dim, idx, cache_l,
+                                         l == ctx->score_layer ? is_new : nullptr, bf.partial, bf.o, ctx->status_dev, st),
+                 "attention_twoseg");
+    } else {
+      mark(ctx, MARCHE_KC_SCATTER_KV, st);
+      MARCHE_TRY(launch_scatter_kv(ctx->bf16, bf.qkv + (size_t)D * eb, bf.qkv + (size_t)2 * D * eb, 3 * D, idx, B, nA,
+                                   S, D, cache_l, st), "scatter_kv");
+      rc = do_attention(ctx, bf.qkv, 3 * D, nA, cache_l, l == ctx->score_layer ? is_new : nullptr, bf.partial, bf.o, st);
+      if (rc) return rc;
+    }
     rc = do_linear(ctx, MARCHE_KC_GEMM_O, bf.o, D, M, bw.w_o, bw.b_o, D, D, MARCHE_EPI_BIAS_RESIDUAL, x, st);
     if (rc) return rc;
     mark(ctx, MARCHE_KC_GATHER_LN, st);
@@ -293,6 +302,8 @@ int marche_create(const marche_config* cfg, const marche_block_weights* blocks, 
   ctx->score_layer = sl;
   const char* fs = getenv("MARCHE_FORCE_SIMT");
   ctx->force_simt = fs && fs[0] == '1';
+  const char* am = getenv("MARCHE_ATTN");
+  ctx->attn_mode = (am && (am[0] == '1' || am[0] == 't')) ? 1 : 0;
   const char* gm = getenv("MARCHE_GEMM");
   ctx->gemm_mode = gm ? atoi(gm) : 0;
   cudaError_t e = cudaGetDevice(&ctx->device);
@@ -467,6 +478,23 @@ int marche_scatter_kv(marche_ctx* ctx, const void* k, const void* v, int ld_kv, 
   return MARCHE_OK;
 }
 
+int marche_attention_two_segment(marche_ctx* ctx, const void* qkv, int ld, int n, const int32_t* active_idx,
+                                 void* cache_layer, const uint8_t* is_new, float* score_partial, void* o,
+                                 marche_stream stream) {
+  if (!ctx || !qkv || !cache_layer || !o || n < 0 || n > ctx->cfg.seq_len || ld < 3 * ctx->cfg.width)
+    return MARCHE_EINVAL;
+  if (!active_idx && n != ctx->cfg.seq_len) return MARCHE_EINVAL;
+  if (is_new && !score_partial) return MARCHE_EINVAL;
+  if (!ctx->bf16) return MARCHE_ESHAPE;
+  if (n == 0) return MARCHE_OK;
+  const marche_config& c = ctx->cfg;
+  mark(ctx, MARCHE_KC_ATTENTION, (cudaStream_t)stream);
+  MARCHE_TRY(launch_attention_twoseg(qkv, ld, c.width, 2 * c.width, c.batch, n, c.seq_len, c.n_heads, c.head_dim,
+                                     active_idx, cache_layer, is_new, score_partial, o, ctx->status_dev,
+                                     (cudaStream_t)stream), "attention_twoseg");
+  return MARCHE_OK;
+}
+
 int marche_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void* cache_layer,
                      const uint8_t* is_new, float* score_partial, void* o, marche_stream stream) {
   if (!ctx || !q || !cache_layer || !o || n < 0 || n > ctx->cfg.seq_len || ld_q < ctx->cfg.width)
@@ -506,7 +534,7 @@ int marche_step_host(marche_ctx* ctx, int full, float* hidden, void* kv_cache, c
     return MARCHE_EINVAL;
   if (((uintptr_t)staging & 255) != 0) return MARCHE_EINVAL;
   if (staging_bytes < marche_staging_bytes(ctx, max_new)) return MARCHE_EWORKSPACE;
-  const size_t B = ctx->cfg.batch, S = ctx->cfg.seq_len, D = ctx->cfg.width, mn = max_new;
+  const size_t B = ctx->cfg.batch, D = ctx->cfg.width, mn = max_new;
   cudaStream_t st = (cudaStream_t)stream;
   char* p = (char*)staging;
   float* d_prev_rows = (float*)p;  p += align256(B * mn * D * sizeof(float));

@@ -202,6 +202,45 @@ def test_attention_and_score_partials(dtype, S, dh, H, n, nG):
     assert (partial2 == -1.0).all()
 
 
+@pytest.mark.parametrize("S", [68, 320, 1088])
+@pytest.mark.parametrize("dh,H", [(64, 4), (80, 8)])
+@pytest.mark.parametrize("n,nG", [(1, 1), (12, 7), (41, 5), (77, 0), (130, 25)])
+def test_two_segment_attention_equals_scatter_then_attend(S, dh, H, n, nG):
+    """The two-segment kernel (Eq. 6-10 + write-back) against the oracle's plain attention over
+    the updated cache, and bit-exact cache contents against marche_scatter_kv."""
+    if n > S:
+        pytest.skip("n > S")
+    B, D = 2, dh * H
+    cfg, blocks, m = model_for("bf16", D, H, 128, S, B)
+    rng = np.random.default_rng(S + n + dh)
+    qkv = (rng.standard_normal((B * n, 3 * D)) * np.array([3.0] * D + [1.0] * 2 * D)).astype(np.float32)
+    cache = rng.standard_normal((2, B, S, D)).astype(np.float32)
+    idx = np.stack([rng.permutation(S)[:n] for _ in range(B)]).astype(np.int32)
+    flags = np.zeros((B, n), dtype=np.uint8)
+    for b in range(B):
+        flags[b, rng.permutation(n)[:nG]] = 1
+    qkv_d = dev(qkv, torch.bfloat16)
+    cache_a, cache_b = dev(cache, torch.bfloat16), dev(cache, torch.bfloat16)
+    o_a = torch.zeros(B * n, D, dtype=torch.float16, device="cuda")
+    p_a = torch.full((B, H, S), -1.0, device="cuda")
+    m.attention_two_segment(qkv_d, 3 * D, n, idx_dev(idx), cache_a, dev(flags), p_a, o_a)
+    m.scatter_kv(qkv_d[:, D:], qkv_d[:, 2 * D:], 3 * D, idx_dev(idx), n, cache_b)
+    torch.cuda.synchronize()
+    assert m.device_status() == 0
+    assert torch.equal(cache_a, cache_b)                               # write-back: byte-identical
+    qq, cc = quant(qkv, "bf16"), host(cache_b)
+    want_o, want_p = np.zeros((B * n, D)), np.zeros((B, H, S))
+    for b in range(B):
+        for h in range(H):
+            c = slice(h * dh, (h + 1) * dh)
+            z, p = orc.softmax_attention(qq[b * n:(b + 1) * n, c], cc[0, b][:, c], cc[1, b][:, c])
+            want_o[b * n:(b + 1) * n, c] = z
+            want_p[b, h] = p[flags[b].astype(bool)].sum(axis=0)
+    assert rel_l2(host(o_a), want_o) <= 8e-3 and max_abs(host(o_a), want_o) <= 3e-2
+    assert max_abs(host(p_a), want_p) <= 2e-2 * max(1, nG) / 8 + 1e-6
+    assert np.allclose(host(p_a).sum(-1), nG, rtol=5e-3, atol=1e-6)
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_attention_uniform_and_peaked(dtype):
     S, B, H, dh, n = 68, 2, 4, 64, 5
