@@ -211,6 +211,20 @@ int marche_select_refresh(marche_ctx* ctx, const float* scores,
                           const int32_t* exclude_idx, int n_excl,
                           int k, int32_t* refresh_idx, void* mask_scratch, marche_stream stream);
 
+/* Selection ablations of Section 5.3 (Table 3): the same call with a policy.  MARCHE_SELECT_HIGH is
+ * the method (highest relevance first); MARCHE_SELECT_LOW picks the lowest scores; and
+ * MARCHE_SELECT_RANDOM ignores the scores and orders the candidates by a 32-bit counter-based hash
+ * of (seed, sample index, token index): x = seed ^ b*0x9E3779B1 ^ t*0x85EBCA77; x ^= x>>16;
+ * x *= 0x7FEB352D; x ^= x>>15; x *= 0x846CA68B; x ^= x>>16 (mod 2^32), smaller first.  Ties go to
+ * the lower token index in every policy.  (The active-set ablations of Table 2 need no kernel: pass
+ * n_prev = 0 or n_new = 0 to marche_build_active.) */
+enum { MARCHE_SELECT_HIGH = 0, MARCHE_SELECT_LOW = 1, MARCHE_SELECT_RANDOM = 2 };
+int marche_select_refresh_policy(marche_ctx* ctx, const float* scores,
+                                 const int32_t* new_idx, int n_new,
+                                 const int32_t* exclude_idx, int n_excl,
+                                 int k, int policy, uint32_t seed, int32_t* refresh_idx,
+                                 void* mask_scratch, marche_stream stream);
+
 /* The same selection as marche_select_refresh for callers that have no scratch buffer to give
  * and cannot obtain one: code running where device allocation is not allowed (inside a region
  * whose memory was sized up front, a latency-critical serving loop that must never touch the

@@ -165,14 +165,27 @@ def fixed_budget_refresh_count(budget: int, n_generating: int, n_caching: int) -
     return max(0, int(budget) - int(n_generating) - int(n_caching))
 
 
+def _mix32(seed: int, b: int, t: int) -> int:
+    """Counter-based 32-bit hash of (seed, sample, token) for the random-selection ablation."""
+    M = 0xFFFFFFFF
+    x = (seed ^ (b * 0x9E3779B1) ^ (t * 0x85EBCA77)) & M
+    x ^= x >> 16
+    x = (x * 0x7FEB352D) & M
+    x ^= x >> 15
+    x = (x * 0x846CA68B) & M
+    x ^= x >> 16
+    return x
+
+
 def select_refresh(scores: np.ndarray, new_idx: np.ndarray, exclude_idx: Optional[np.ndarray],
-                   k: int) -> np.ndarray:
+                   k: int, policy: str = "high", seed: int = 0) -> np.ndarray:
     """Section 4.2: the k candidate tokens with the highest relevance score.
 
     scores fp32 [B][S].  Candidates are all tokens not in new_idx[b] or
     exclude_idx[b].  Reading (the paper gives no tie rule): rank by score
     descending, then token index ascending; the result is int32 [B][k] in
-    ascending index order.  Done by a full sort."""
+    ascending index order.  Done by a full sort.  `policy` "low" / "random" are the selection
+    ablations of Section 5.3 (lowest scores first; order by a hash of seed, sample and token)."""
     scores = np.asarray(scores, dtype=np.float32)
     B, S = scores.shape
     out = np.zeros((B, k), dtype=np.int32)
@@ -183,7 +196,14 @@ def select_refresh(scores: np.ndarray, new_idx: np.ndarray, exclude_idx: Optiona
         cand = [t for t in range(S) if t not in banned]
         if k > len(cand):
             raise ValueError("k exceeds the number of candidates")
-        ranked = sorted(cand, key=lambda t: (-float(scores[b, t]), t))
+        if policy == "high":            # the method: highest relevance first
+            ranked = sorted(cand, key=lambda t: (-float(scores[b, t]), t))
+        elif policy == "low":           # ablation (Section 5.3): lowest attention first
+            ranked = sorted(cand, key=lambda t: (float(scores[b, t]) + 0.0, t))
+        elif policy == "random":        # ablation: random candidates
+            ranked = sorted(cand, key=lambda t: (_mix32(seed, b, t), t))
+        else:
+            raise ValueError("unknown policy")
         out[b] = np.array(sorted(ranked[:k]), dtype=np.int32)
     return out
 

@@ -51,6 +51,7 @@ _SIGNATURES = {
     "marche_full_step": (C.c_int, [_vp, _vp, _vp, _vp, _i, _vp, _i, _f, _vp, _vp, C.POINTER(C.c_int), _vp, _sz, _vp]),
     "marche_step_in_step_selection": (C.c_int, [_vp, _vp, _vp, _vp, _i, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "marche_select_refresh": (C.c_int, [_vp, _vp, _vp, _i, _vp, _i, _i, _vp, _vp, _vp]),
+    "marche_select_refresh_policy": (C.c_int, [_vp, _vp, _vp, _i, _vp, _i, _i, _i, C.c_uint32, _vp, _vp, _vp]),
     "marche_select_refresh_static": (C.c_int, [_vp, _vp, _vp, _i, _vp, _i, _i, _vp, _vp]),
     "marche_get_scores": (C.c_int, [_vp, _vp, _vp, _vp]),
     "marche_build_active": (C.c_int, [_vp, _vp, _i, _vp, _i, _vp, _i, _vp, _vp]),
@@ -220,6 +221,14 @@ class Marche:
         self._check(self.lib.marche_select_refresh(
             self.h, _ptr(scores), _ptr(new_idx), 0 if new_idx is None else new_idx.shape[1],
             _ptr(exclude_idx), 0 if exclude_idx is None else exclude_idx.shape[1], k, _ptr(refresh_idx),
+            _ptr(mask_scratch), _stream(stream)))
+
+    def select_refresh_policy(self, scores, new_idx, exclude_idx, k, policy, seed, refresh_idx, mask_scratch,
+                              stream=None):
+        """policy 0 = highest scores (the method), 1 = lowest scores, 2 = random (hash of seed, sample, token)."""
+        self._check(self.lib.marche_select_refresh_policy(
+            self.h, _ptr(scores), _ptr(new_idx), 0 if new_idx is None else new_idx.shape[1],
+            _ptr(exclude_idx), 0 if exclude_idx is None else exclude_idx.shape[1], k, policy, seed, _ptr(refresh_idx),
             _ptr(mask_scratch), _stream(stream)))
 
     def select_refresh_static(self, scores, new_idx, exclude_idx, k, refresh_idx, stream=None):

@@ -388,7 +388,15 @@ int marche_step_in_step_selection(marche_ctx* ctx, const float* hidden, void* kv
 int marche_select_refresh(marche_ctx* ctx, const float* scores, const int32_t* new_idx, int n_new,
                           const int32_t* exclude_idx, int n_excl, int k, int32_t* refresh_idx, void* mask_scratch,
                           marche_stream stream) {
+  return marche_select_refresh_policy(ctx, scores, new_idx, n_new, exclude_idx, n_excl, k, MARCHE_SELECT_HIGH, 0u,
+                                      refresh_idx, mask_scratch, stream);
+}
+
+int marche_select_refresh_policy(marche_ctx* ctx, const float* scores, const int32_t* new_idx, int n_new,
+                                 const int32_t* exclude_idx, int n_excl, int k, int policy, uint32_t seed,
+                                 int32_t* refresh_idx, void* mask_scratch, marche_stream stream) {
   if (!ctx || !scores || !mask_scratch || n_new < 0 || n_excl < 0 || k < 0) return MARCHE_EINVAL;
+  if (policy < MARCHE_SELECT_HIGH || policy > MARCHE_SELECT_RANDOM) return MARCHE_EINVAL;
   if ((n_new > 0 && !new_idx) || (n_excl > 0 && !exclude_idx)) return MARCHE_EINVAL;
   const int B = ctx->cfg.batch, S = ctx->cfg.seq_len;
   if (k > S - n_new - n_excl) return MARCHE_EINVAL;
@@ -400,7 +408,7 @@ int marche_select_refresh(marche_ctx* ctx, const float* scores, const int32_t* n
                                st), "flags");
   mark(ctx, MARCHE_KC_TOPK, st);
   MARCHE_TRY(launch_topk(nullptr, 0, const_cast<float*>(scores), (const uint8_t*)mask_scratch, B, S, k, refresh_idx,
-                         st), "topk");
+                         st, policy, seed), "topk");
   return MARCHE_OK;
 }
 

@@ -22,9 +22,22 @@ MARCHE_DEVINL uint32_t score_key(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// Counter-based 32-bit mix of (seed, sample, token) for the random-selection ablation: xor the
+// three words with odd multipliers, then two xorshift-multiply rounds.
+MARCHE_DEVINL uint32_t mix32(uint32_t seed, uint32_t b, uint32_t t) {
+  uint32_t x = seed ^ (b * 0x9E3779B1u) ^ (t * 0x85EBCA77u);
+  x ^= x >> 16; x *= 0x7FEB352Du;
+  x ^= x >> 15; x *= 0x846CA68Bu;
+  x ^= x >> 16;
+  return x;
+}
+
+// policy 0: highest score first (Section 4.2); 1: lowest score first and 2: random order (the
+// selection ablations of Section 5.3).  Ties always go to the lower token index.
 __global__ void __launch_bounds__(kTopkThreads)
 topk_kernel(const float* __restrict__ partial, int H, float* __restrict__ scores,
-            const uint8_t* __restrict__ cand, int S, int k, int32_t* __restrict__ refresh_idx) {
+            const uint8_t* __restrict__ cand, int S, int k, int policy, uint32_t seed,
+            int32_t* __restrict__ refresh_idx) {
   extern __shared__ unsigned long long comp[];          // [S] composite keys; 0 = not a candidate
   __shared__ int warp_tot[kTopkThreads / 32];
   const int b = blockIdx.x, tid = threadIdx.x;
@@ -41,8 +54,9 @@ topk_kernel(const float* __restrict__ partial, int H, float* __restrict__ scores
     }
     // composite key: score key in the high word, reversed index in the low word, so a
     // larger composite means "ranked earlier" and all composites are distinct and > 0.
+    const uint32_t key = policy == 0 ? score_key(s) : (policy == 1 ? ~score_key(s) : ~mix32(seed, (uint32_t)b, (uint32_t)t));
     comp[t] = (k > 0 && cand[(long)b * S + t])
-                  ? (((unsigned long long)score_key(s) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)t))
+                  ? (((unsigned long long)key << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)t))
                   : 0ull;
   }
   if (k <= 0) return;
@@ -83,10 +97,10 @@ topk_kernel(const float* __restrict__ partial, int H, float* __restrict__ scores
 }
 
 cudaError_t launch_topk(const float* partial, int H, float* scores, const uint8_t* cand, int B, int S, int k,
-                        int32_t* refresh_idx, cudaStream_t st) {
+                        int32_t* refresh_idx, cudaStream_t st, int policy, uint32_t seed) {
   if (S > 2048) return cudaErrorInvalidValue;
   return launch_pdl(topk_kernel, dim3(B), dim3(kTopkThreads), (size_t)S * sizeof(unsigned long long), st, partial, H,
-                    scores, cand, S, k, refresh_idx);
+                    scores, cand, S, k, policy, seed, refresh_idx);
 }
 
 }  // namespace marche

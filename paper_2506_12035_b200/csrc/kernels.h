@@ -39,8 +39,9 @@ cudaError_t launch_validate(const int32_t* active_idx, int n_active, const int32
 
 // K4: optional fixed-order head reduction of score partials [B][H][S] into scores [B][S],
 // then top-k among cand (k may be 0: reduction only).
+// policy 0 = highest scores, 1 = lowest scores, 2 = random (counter-based hash of seed, sample, token).
 cudaError_t launch_topk(const float* partial, int H, float* scores, const uint8_t* cand, int B, int S, int k,
-                        int32_t* refresh_idx, cudaStream_t st);
+                        int32_t* refresh_idx, cudaStream_t st, int policy = 0, uint32_t seed = 0);
 
 // K2 (fp32 SIMT and bf16 SIMT bring-up path).
 cudaError_t launch_gemm_simt(bool bf16_t, const void* a, int lda, int M, const void* w, const float* bias,

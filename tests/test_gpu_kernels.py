@@ -295,6 +295,21 @@ def test_select_refresh_bit_exact(S, k):
                 assert (out.cpu().numpy() == -1).all()
 
 
+@pytest.mark.parametrize("policy,name", [(0, "high"), (1, "low"), (2, "random")])
+def test_select_refresh_policies_bit_exact(policy, name):
+    B, S, k = 5, 320, 32
+    cfg, blocks, m = model_for("f32", 128, 2, 128, S, B)
+    rng = np.random.default_rng(policy)
+    mask = torch.empty(B * S, dtype=torch.uint8, device="cuda")
+    for sc in (rng.random((B, S)), rng.integers(0, 4, (B, S)).astype(float), np.zeros((B, S))):
+        sc = sc.astype(np.float32)
+        perm = np.stack([rng.permutation(S) for _ in range(B)]).astype(np.int32)
+        new, excl = perm[:, :4], perm[:, 4:9]
+        out = torch.full((B, k), -1, dtype=torch.int32, device="cuda")
+        m.select_refresh_policy(dev(sc), idx_dev(new), idx_dev(excl), k, policy, 1234, out, mask)
+        assert np.array_equal(out.cpu().numpy(), orc.select_refresh(sc, new, excl, k, policy=name, seed=1234))
+
+
 def test_validate_indices():
     from paper_2506_12035_b200.binding import MarcheError
     S, B = 68, 2

@@ -441,6 +441,31 @@ def test_P10_topk_vs_stable_argsort(S, k):
             assert got[b].tolist() == sorted(order[:k].tolist())
 
 
+def test_selection_ablation_policies():
+    rng = np.random.default_rng(11)
+    S, B, k = 40, 3, 6
+    sc = rng.random((B, S)).astype(np.float32)
+    new = np.stack([rng.permutation(S)[:3] for _ in range(B)]).astype(np.int32)
+    hi = orc.select_refresh(sc, new, None, k, policy="high")
+    lo = orc.select_refresh(sc, new, None, k, policy="low")
+    for b in range(B):
+        cand = [t for t in range(S) if t not in set(new[b].tolist())]
+        assert sorted(sorted(cand, key=lambda t: sc[b, t])[:k]) == lo[b].tolist()
+        assert sc[b, lo[b]].max() < sc[b, hi[b]].min()
+    # low policy == high policy on negated scores (distinct values)
+    assert np.array_equal(lo, orc.select_refresh(1.0 - sc, new, None, k, policy="high"))
+    r1 = orc.select_refresh(sc, new, None, k, policy="random", seed=5)
+    r2 = orc.select_refresh(sc * 0, new, None, k, policy="random", seed=5)
+    r3 = orc.select_refresh(sc, new, None, k, policy="random", seed=6)
+    assert np.array_equal(r1, r2) and not np.array_equal(r1, r3)          # scores ignored, seed matters
+    for b in range(B):
+        assert not set(r1[b].tolist()) & set(new[b].tolist()) and len(set(r1[b].tolist())) == k
+    # the hash spreads: over many tokens the selected fraction per half is balanced
+    big = orc.select_refresh(np.zeros((1, 1000), np.float32), np.zeros((1, 0), np.int32), None, 500, policy="random", seed=1)
+    assert 200 < (big[0] < 500).sum() < 300
+    assert orc._mix32(0, 0, 0) == 0 and orc._mix32(1, 2, 3) == orc._mix32(1, 2, 3) and orc._mix32(1, 2, 3) != orc._mix32(1, 3, 2)
+
+
 def test_topk_signed_zero_and_errors():
     sc = np.array([[0.0, -0.0, 0.0, -0.0]], dtype=np.float32)
     assert orc.select_refresh(sc, np.zeros((1, 0), np.int32), None, 2).tolist() == [[0, 1]]
