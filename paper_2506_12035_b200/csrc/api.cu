@@ -33,6 +33,8 @@ struct marche_ctx {
   float eps = 1e-6f;
   int score_layer = 0;
   bool force_simt = false;
+  int attn_tc = -1;                                   // -1 auto, 0 never, 1 always (MARCHE_ATTN_TC)
+  int attn_tc_min_rows = 96;                          // auto: tcgen05 attention above this many active rows
   int attn_mode = 0;                                  // 0 write-back kernel + one-segment attention, 1 two-segment (MARCHE_ATTN)
   int gemm_mode = 0;                                  // 0 auto, 1 single-CTA MMA, 2 CTA-pair MMA (MARCHE_GEMM)
   std::vector<std::pair<const void*, bool>> caches;  // (cache pointer, filled)
@@ -125,7 +127,18 @@ int do_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void* ca
   if (n > 0) mark(ctx, MARCHE_KC_ATTENTION, st);
   const bool tc = ctx->bf16 && !ctx->force_simt && (c.head_dim == 64 || c.head_dim == 80) && ld_q % 2 == 0 &&
                   ((uintptr_t)q & 3) == 0 && ((uintptr_t)cache_layer & 15) == 0;
-  if (tc)
+  // Two tensor-core kernels.  At small active sets the step is bound by streaming the cache and the
+  // mma.sync kernel (several small CTAs per SM, one pass) is faster: 41 us vs 69 us at n = 41.  Once
+  // the legacy tensor path saturates (about 250 TFLOP/s) the tcgen05 kernel wins: 109 vs 172 us at
+  // n = 122 (S 1088), 840 vs 1100 us at n = S = 1088, and earlier for the two-pass scoring flavour
+  // (97 vs 143 us at n = 77).  MARCHE_ATTN_TC=0 / 1 forces one of them; head_dim 80 has only the former.
+  const int tc_min = is_new ? 64 : ctx->attn_tc_min_rows;
+  const bool tc5 = tc && c.head_dim == 64 && ld_q % 8 == 0 && ((uintptr_t)q & 15) == 0 &&
+                   (ctx->attn_tc == 1 || (ctx->attn_tc < 0 && n > tc_min));
+  if (tc5)
+    MARCHE_TRY(launch_attention_tcgen05(q, ld_q, c.batch, n, c.seq_len, c.n_heads, c.head_dim, cache_layer, is_new,
+                                        partial, o, ctx->status_dev, st), "attention_tcgen05");
+  else if (tc)
     MARCHE_TRY(launch_attention_mma(q, ld_q, c.batch, n, c.seq_len, c.n_heads, c.head_dim, cache_layer, is_new,
                                     partial, o, ctx->status_dev, st), "attention_mma");
   else
@@ -302,6 +315,10 @@ int marche_create(const marche_config* cfg, const marche_block_weights* blocks, 
   ctx->score_layer = sl;
   const char* fs = getenv("MARCHE_FORCE_SIMT");
   ctx->force_simt = fs && fs[0] == '1';
+  const char* tcv = getenv("MARCHE_ATTN_TC");
+  if (tcv) ctx->attn_tc = atoi(tcv);
+  const char* tcm = getenv("MARCHE_ATTN_TC_MIN");
+  if (tcm) ctx->attn_tc_min_rows = atoi(tcm);
   const char* am = getenv("MARCHE_ATTN");
   ctx->attn_mode = (am && (am[0] == '1' || am[0] == 't')) ? 1 : 0;
   const char* gm = getenv("MARCHE_GEMM");

@@ -69,6 +69,12 @@ cudaError_t launch_attention_mma(const void* q, int ld_q, int B, int n, int S, i
                                  const void* cache_layer, const uint8_t* is_new, float* score_partial, void* o,
                                  int* status, cudaStream_t st);
 
+// K3 on tcgen05 (head_dim 64 only): S = Q K^T and O = P V as tcgen05.mma with TMEM accumulators.
+// ld_q % 8 == 0; q and cache_layer 16-byte aligned.
+cudaError_t launch_attention_tcgen05(const void* q, int ld_q, int B, int n, int S, int H, int dh,
+                                     const void* cache_layer, const uint8_t* is_new, float* score_partial, void* o,
+                                     int* status, cudaStream_t st);
+
 // K3, two-segment flavour (Eq. 6-10 without concatenation, then the cache write-back of Algorithm 1
 // line 11 by the same kernel): fresh K/V are columns k_off / v_off of the compact qkv buffer
 // [B*n][ld]; active_idx NULL = identity.  Same type and alignment rules as launch_attention_mma.
