@@ -33,6 +33,8 @@ struct marche_ctx {
   float eps = 1e-6f;
   int score_layer = 0;
   bool force_simt = false;
+  bool fuse_writeback = false;                        // MARCHE_FUSE_WB=1: write-back fused into the attention prologue
+                                                      // (measured slower: +11.7 us attention vs -10.5 us scatter_kv launch)
   int attn_tc = -1;                                   // -1 auto, 0 never, 1 always (MARCHE_ATTN_TC)
   int attn_tc_min_rows = 96;                          // auto: tcgen05 attention above this many active rows
   int attn_mode = 0;                                  // 0 write-back kernel + one-segment attention, 1 two-segment (MARCHE_ATTN)
@@ -197,6 +199,14 @@ int run_blocks(marche_ctx* ctx, int l_begin, int l_end, const float* gather_src,
       MARCHE_TRY(launch_attention_twoseg(bf.qkv, 3 * D, D, 2 * D, B, nA, S, c.n_heads, c.head_dim, idx, cache_l,
                                          l == ctx->score_layer ? is_new : nullptr, bf.partial, bf.o, ctx->status_dev, st),
                  "attention_twoseg");
+    } else if (ctx->fuse_writeback && ctx->bf16 && !ctx->force_simt && ctx->attn_tc != 1 &&
+               !(c.head_dim == 64 && ctx->attn_tc < 0 &&
+                 nA > ((l == ctx->score_layer && is_new) ? 64 : ctx->attn_tc_min_rows))) {
+      // mma.sync attention with the cache write-back fused into its prologue (no scatter_kv launch)
+      mark(ctx, MARCHE_KC_ATTENTION, st);
+      MARCHE_TRY(launch_attention_mma(bf.qkv, 3 * D, B, nA, S, c.n_heads, c.head_dim, cache_l,
+                                      l == ctx->score_layer ? is_new : nullptr, bf.partial, bf.o, ctx->status_dev, st,
+                                      true, idx, D, 2 * D), "attention_mma_wb");
     } else {
       mark(ctx, MARCHE_KC_SCATTER_KV, st);
       MARCHE_TRY(launch_scatter_kv(ctx->bf16, bf.qkv + (size_t)D * eb, bf.qkv + (size_t)2 * D * eb, 3 * D, idx, B, nA,
@@ -315,6 +325,8 @@ int marche_create(const marche_config* cfg, const marche_block_weights* blocks, 
   ctx->score_layer = sl;
   const char* fs = getenv("MARCHE_FORCE_SIMT");
   ctx->force_simt = fs && fs[0] == '1';
+  const char* fw = getenv("MARCHE_FUSE_WB");
+  ctx->fuse_writeback = fw && fw[0] == '1';
   const char* tcv = getenv("MARCHE_ATTN_TC");
   if (tcv) ctx->attn_tc = atoi(tcv);
   const char* tcm = getenv("MARCHE_ATTN_TC_MIN");

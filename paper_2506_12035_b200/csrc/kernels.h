@@ -65,9 +65,13 @@ size_t attention_simt_smem(int S, int dh);
 
 // K3 (bf16, TMA-staged K/V tiles, tensor-core QK^T and PV, fused score column sums).
 // head_dim 64 or 80; ld_q even; cache_layer 16-byte aligned.
+// write_back: each CTA first copies its head's fresh K / V rows (columns k_off / v_off relative to q,
+// same row stride; token of row j = wb_idx[b][j], nullptr = identity) into cache_layer, replacing a
+// separate launch_scatter_kv (needs ld_q % 8 == 0 and q 16-byte aligned).
 cudaError_t launch_attention_mma(const void* q, int ld_q, int B, int n, int S, int H, int dh,
                                  const void* cache_layer, const uint8_t* is_new, float* score_partial, void* o,
-                                 int* status, cudaStream_t st);
+                                 int* status, cudaStream_t st, bool write_back = false, const int32_t* wb_idx = nullptr,
+                                 int k_off = 0, int v_off = 0);
 
 // K3 on tcgen05 (head_dim 64 only): S = Q K^T and O = P V as tcgen05.mma with TMEM accumulators.
 // ld_q % 8 == 0; q and cache_layer 16-byte aligned.
