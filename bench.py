@@ -52,6 +52,23 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
+# ----------------------------------------------------------------------------- replicas (N > 1)
+def max_over_ranks(value: float, device="cuda") -> float:
+    """The slowest rank's time: with N independent replicas the job is as slow as its slowest GPU."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_images_per_s(n_images_per_rank: int, ms_max: float, world: int) -> float:
+    """Whole-job throughput of `world` replicas that each generate n_images_per_rank images."""
+    return world * n_images_per_rank / (ms_max * 1e-3)
+
+
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -279,10 +296,7 @@ def run_ours(args, cfg):
             fn()
         e1.record()
         barrier()
-        ms = torch.tensor([e0.elapsed_time(e1)], device="cuda")
-        if world > 1:
-            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        return float(ms.item()) / reps
+        return max_over_ranks(e0.elapsed_time(e1)) / reps
 
     n_dec = args.decode_steps or None
     for _ in range(args.warmup):
@@ -295,7 +309,7 @@ def run_ours(args, cfg):
     launches = m.launch_count() - launches0
     clock_info = clocks.stop()
     assert m.device_status() == 0, "a bounded device wait gave up"
-    value = world * n_images / (ms_gen * 1e-3)
+    value = aggregate_images_per_s(n_images, ms_gen, world)
 
     line = {"metric": METRIC, "value": value, "unit": "images/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_gen, "higher_is_better": True, "scaling": "weak",
