@@ -98,7 +98,10 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
   ptx::cluster_sync_all();                                // both CTAs' barriers exist before any remote signal
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  pdl_sync();                                             // set-up above overlaps the previous kernel's tail
+  // Programmatic dependent launch: everything above overlapped the previous kernel's tail.  The
+  // producer additionally fetches the first weight tiles (weights are never written by a kernel)
+  // before it waits for the previous kernel; every other thread waits right here.
+  if (!(warp == 0 && lane == 0)) pdl_sync();
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer (both CTAs)
@@ -106,6 +109,17 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       ptx::prefetch_tensormap(&tmap_a);
       ptx::prefetch_tensormap(&tmap_w);
       ptx::prefetch_tensormap(&tmap_out);
+      int prefetched = 0;                                  // ring slots whose barrier is armed and W half loaded
+      if (pair < n_tiles) {
+        const int n_blk0 = pair % n_n;
+        const int wrow0 = n_blk0 * BN + (int)rank * (BN / 2);
+        for (; prefetched < STAGES && prefetched < n_kb; ++prefetched) {
+          const uint32_t leader_full = ptx::mapa(full_bar(prefetched), 0);
+          if (rank == 0) ptx::mbar_expect_tx(full_bar(prefetched), 2 * Cfg::STAGE_BYTES);
+          ptx::tma_load_2d_pair(w_tile(prefetched), &tmap_w, prefetched * BK, wrow0, leader_full);
+        }
+      }
+      pdl_sync();
       int it = 0;
       bool ok = true;
       for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
@@ -114,9 +128,13 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
         const int wrow0 = n_blk * BN + (int)rank * (BN / 2);          // this CTA's half of the W tile
         for (int kb = 0; kb < n_kb; ++kb, ++it) {
           const int s = it % STAGES;
+          const uint32_t leader_full = ptx::mapa(full_bar(s), 0);
+          if (it < prefetched) {                           // slot armed and W already in flight
+            ptx::tma_load_2d_pair(a_tile(s), &tmap_a, kb * BK, row0, leader_full);
+            continue;
+          }
           const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
           if (!ptx::mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
-          const uint32_t leader_full = ptx::mapa(full_bar(s), 0);
           if (rank == 0) ptx::mbar_expect_tx(full_bar(s), 2 * Cfg::STAGE_BYTES);
           ptx::tma_load_2d_pair(a_tile(s), &tmap_a, kb * BK, row0, leader_full);
           ptx::tma_load_2d_pair(w_tile(s), &tmap_w, kb * BK, wrow0, leader_full);
@@ -180,7 +198,8 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa(tempty_bar(acc), 0));
     }
     if (!ok && lane == 0) *(volatile int*)status = ST2_EPILOGUE;
-    if (lane == 0) ptx::bulk_wait_all();                    // this warp's stores have left shared memory and landed
+    if (lane == 0) ptx::bulk_wait_read_all();               // the TMA engine has read this warp's staging box;
+                                                            // the writes complete with the grid
   }
 
   ptx::tc_fence_before();
