@@ -33,6 +33,7 @@ struct marche_ctx {
   float eps = 1e-6f;
   int score_layer = 0;
   bool force_simt = false;
+  bool stream_k = true;                               // MARCHE_STREAM_K=0: whole tiles only in the residual GEMMs
   bool fuse_writeback = false;                        // MARCHE_FUSE_WB=1: write-back fused into the attention prologue
                                                       // (measured slower: +11.7 us attention vs -10.5 us scatter_kv launch)
   int attn_tc = -1;                                   // -1 auto, 0 never, 1 always (MARCHE_ATTN_TC)
@@ -55,7 +56,7 @@ namespace {
 inline size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 struct WsLayout {
-  size_t scores, partial, cand, is_new, x, x2, u, qkv, o, g, total;
+  size_t scores, partial, cand, is_new, turn, turn_bytes, x, x2, u, qkv, o, g, total;
 };
 
 WsLayout ws_layout(const marche_ctx* c, int nA) {
@@ -67,6 +68,8 @@ WsLayout ws_layout(const marche_ctx* c, int nA) {
   w.partial = off; off += align256(B * H * S * sizeof(float));
   w.cand = off;    off += align256(B * S);
   w.is_new = off;  off += align256(M);
+  w.turn_bytes = gemm_tcgen05_2cta_turn_bytes((int)M, (int)D);   // stream-K turn flags of the residual GEMMs
+  w.turn = off;    off += align256(w.turn_bytes);
   w.x = off;       off += align256(M * D * sizeof(float));
   w.x2 = off;      off += align256(M * D * sizeof(float));   // second residual buffer (in-step selection)
   w.u = off;       off += align256(M * D * eb);
@@ -109,13 +112,14 @@ int refresh_count(float ratio, int S, int n_cand) {
 }
 
 int do_linear(marche_ctx* ctx, int cls, const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
-              int epi, void* out, cudaStream_t st) {
+              int epi, void* out, cudaStream_t st, int* turn = nullptr) {
   if (M > 0) mark(ctx, cls, st);
   const bool tc = ctx->bf16 && !ctx->force_simt && N % 128 == 0 && K % 64 == 0 && lda % 8 == 0 &&
                   (((uintptr_t)a | (uintptr_t)w | (uintptr_t)out) & 15) == 0;
   const bool pair = tc && (ctx->gemm_mode == 2 || (ctx->gemm_mode == 0 && M > 128));
   if (pair)
-    MARCHE_TRY(launch_gemm_tcgen05_2cta(a, lda, M, w, bias, N, K, epi, out, ctx->status_dev, st), "gemm_tcgen05_2cta");
+    MARCHE_TRY(launch_gemm_tcgen05_2cta(a, lda, M, w, bias, N, K, epi, out, ctx->status_dev, st,
+                                        ctx->stream_k ? turn : nullptr), "gemm_tcgen05_2cta");
   else if (tc)
     MARCHE_TRY(launch_gemm_tcgen05(a, lda, M, w, bias, N, K, epi, out, ctx->status_dev, st), "gemm_tcgen05");
   else
@@ -152,6 +156,7 @@ int do_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void* ca
 struct StackBufs {
   float* scores; float* partial; uint8_t* cand; uint8_t* is_new;
   float* x; float* x2; char* u; char* qkv; char* o; char* g;
+  int* turn;
 };
 
 StackBufs carve(void* workspace, const WsLayout& w) {
@@ -161,6 +166,7 @@ StackBufs carve(void* workspace, const WsLayout& w) {
   b.partial = (float*)(ws + w.partial);
   b.cand = (uint8_t*)(ws + w.cand);
   b.is_new = (uint8_t*)(ws + w.is_new);
+  b.turn = (int*)(ws + w.turn);
   b.x = (float*)(ws + w.x);
   b.x2 = (float*)(ws + w.x2);
   b.u = ws + w.u;
@@ -214,14 +220,14 @@ int run_blocks(marche_ctx* ctx, int l_begin, int l_end, const float* gather_src,
       rc = do_attention(ctx, bf.qkv, 3 * D, nA, cache_l, l == ctx->score_layer ? is_new : nullptr, bf.partial, bf.o, st);
       if (rc) return rc;
     }
-    rc = do_linear(ctx, MARCHE_KC_GEMM_O, bf.o, D, M, bw.w_o, bw.b_o, D, D, MARCHE_EPI_BIAS_RESIDUAL, x, st);
+    rc = do_linear(ctx, MARCHE_KC_GEMM_O, bf.o, D, M, bw.w_o, bw.b_o, D, D, MARCHE_EPI_BIAS_RESIDUAL, x, st, bf.turn);
     if (rc) return rc;
     mark(ctx, MARCHE_KC_GATHER_LN, st);
     MARCHE_TRY(launch_gather_layernorm(ctx->bf16, x, nA, nullptr, B, nA, D, bw.ln2_g, bw.ln2_b, ctx->eps, nullptr,
                                        bf.u, st), "layernorm2");
     rc = do_linear(ctx, MARCHE_KC_GEMM_FC1, bf.u, D, M, bw.w_fc1, bw.b_fc1, F, D, MARCHE_EPI_BIAS_GELU, bf.g, st);
     if (rc) return rc;
-    rc = do_linear(ctx, MARCHE_KC_GEMM_FC2, bf.g, F, M, bw.w_fc2, bw.b_fc2, D, F, MARCHE_EPI_BIAS_RESIDUAL, x, st);
+    rc = do_linear(ctx, MARCHE_KC_GEMM_FC2, bf.g, F, M, bw.w_fc2, bw.b_fc2, D, F, MARCHE_EPI_BIAS_RESIDUAL, x, st, bf.turn);
     if (rc) return rc;
   }
   return MARCHE_OK;
@@ -244,6 +250,8 @@ int run_stack(marche_ctx* ctx, const float* hidden, void* kv_cache, const int32_
   if (n_refresh) *n_refresh = k;
   const StackBufs bf = carve(workspace, w);
 
+  // the workspace is scratch between calls: make sure the stream-K turn flags start at zero
+  if (ctx->bf16 && ctx->stream_k) MARCHE_TRY(cudaMemsetAsync(bf.turn, 0, w.turn_bytes, st), "memset");
   mark(ctx, MARCHE_KC_FLAGS, st);
   MARCHE_TRY(launch_step_flags(active_idx, nA, new_idx, n_new, excl_idx, n_excl, B, S, bf.is_new, bf.cand, st), "flags");
   const int rc = run_blocks(ctx, 0, L, hidden, S, active_idx, nA, bf.x, bf, kv_cache, bf.is_new, st);
@@ -272,6 +280,7 @@ int run_in_step(marche_ctx* ctx, const float* hidden, void* kv_cache, const int3
   if (ws_bytes < w.total) return MARCHE_EWORKSPACE;
   const StackBufs bf = carve(workspace, w);
   const int nA = n_new + n_prev + k;
+  if (ctx->bf16 && ctx->stream_k) MARCHE_TRY(cudaMemsetAsync(bf.turn, 0, w.turn_bytes, st), "memset");
 
   // phase 1: every token; generating rows flagged for the scores; candidates = all \ (new u prev)
   mark(ctx, MARCHE_KC_FLAGS, st);
@@ -325,6 +334,8 @@ int marche_create(const marche_config* cfg, const marche_block_weights* blocks, 
   ctx->score_layer = sl;
   const char* fs = getenv("MARCHE_FORCE_SIMT");
   ctx->force_simt = fs && fs[0] == '1';
+  const char* sk = getenv("MARCHE_STREAM_K");
+  ctx->stream_k = !(sk && sk[0] == '0');
   const char* fw = getenv("MARCHE_FUSE_WB");
   ctx->fuse_writeback = fw && fw[0] == '1';
   const char* tcv = getenv("MARCHE_ATTN_TC");

@@ -13,7 +13,8 @@
 namespace marche {
 
 // Columns covered per call: 32 (EPI 1) or 64 (EPI 0, 2), starting at TMEM column t_col / output
-// column `col`.  stage = this warp's 4 KB box (1024-byte aligned shared address).
+// column `col`.  stage = this warp's 4 KB box (1024-byte aligned shared address).  bias_col may be
+// nullptr for EPI 1 (a partial sum of a split K range whose bias another piece adds).
 template <int EPI>
 MARCHE_DEVINL void epilogue_box(uint32_t t_addr, const float* __restrict__ bias_col, const CUtensorMap* out_map,
                                 int col, int row0, uint32_t stage, int lane) {
@@ -28,7 +29,7 @@ MARCHE_DEVINL void epilogue_box(uint32_t t_addr, const float* __restrict__ bias_
     ptx::tmem_ld_wait();
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      const float4 bv = __ldg(b4 + j);
+      const float4 bv = bias_col ? __ldg(b4 + j) : make_float4(0.f, 0.f, 0.f, 0.f);
       const uint32_t dst = row_base + (uint32_t)((j ^ (lane & 7)) << 4);
       asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(__uint_as_float(r[4 * j + 0]) + bv.x),
                    "f"(__uint_as_float(r[4 * j + 1]) + bv.y), "f"(__uint_as_float(r[4 * j + 2]) + bv.z),

@@ -53,8 +53,11 @@ cudaError_t launch_gemm_tcgen05(const void* a, int lda, int M, const void* w, co
                                 int epilogue, void* out, int* status, cudaStream_t st);
 int gemm_tcgen05_pick_bn(int M, int N);
 // Same contract, tcgen05.mma cta_group::2: CTA pairs share 256 x BN tiles (cluster of 2, no multicast).
+// `turn`: optional zero-filled device scratch of gemm_tcgen05_2cta_turn_bytes(M, N) bytes; with it the
+// residual epilogue may use stream-K (ordered reduce-adds; the flags are left zero again).
 cudaError_t launch_gemm_tcgen05_2cta(const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
-                                     int epilogue, void* out, int* status, cudaStream_t st);
+                                     int epilogue, void* out, int* status, cudaStream_t st, int* turn = nullptr);
+size_t gemm_tcgen05_2cta_turn_bytes(int M, int N);
 int gemm_tcgen05_2cta_pick_bn(int M, int N);
 
 // K3 (SIMT): attention of n queries per sample over all S cache rows.
