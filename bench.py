@@ -343,6 +343,10 @@ def run_ours(args, cfg):
                             "peak_source": "%s (%s)" % (peak_kind, "sustained bf16 GEMM" if dom["bound"] == "tensor" else "device copy"),
                             "timing": "CUDA events in front of every launch, cache-aware steps of one generation of the timed workload"}
 
+        # ---- each kernel on its own at the median cache-aware shape (no dependency gaps)
+        n_mid = int(np.median([s_[1] for s_ in sched[1:]]))
+        line["kernels_isolated"] = {"n_active": n_mid, "rows": isolated_kernels(m, cfg, peaks, n_mid)}
+
         # ---- this build's own full-recompute path (full step at every decoding step)
         gen.run(hidden0, mode="full")
         ms_full = timed(lambda: gen.run(hidden0, mode="full"), 1)
@@ -377,6 +381,69 @@ def run_ours(args, cfg):
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def isolated_kernels(m, cfg, peaks, n_active):
+    """Each hot-path kernel timed on its own at one mid-run shape (n_active rows per sample):
+    back-to-back launches through the single-kernel C calls, CUDA events around the batch, buffers
+    rotated so that streamed operands come from HBM.  Unlike the per-class table of the generation,
+    these figures contain no dependency gaps: they are the kernels' own roofline fractions."""
+    import torch
+    B, S, D, F, H = cfg.B, cfg.S, cfg.D, cfg.F, cfg.H
+    M = B * n_active
+    dev = "cuda"
+    act = torch.float16 if cfg.dtype == "bf16" else torch.float32
+    typ = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    eb = 2 if cfg.dtype == "bf16" else 4
+    rot = 3
+    xs = [torch.randn(M, D, device=dev) for _ in range(rot)]
+    us = [torch.empty(M, D, device=dev, dtype=act) for _ in range(rot)]
+    qkvs = [torch.randn(M, 3 * D, device=dev).to(typ) for _ in range(rot)]
+    caches = [torch.randn(2, B, S, D, device=dev).to(typ) for _ in range(rot)]
+    o = torch.empty(M, D, device=dev, dtype=act)
+    g = torch.empty(M, F, device=dev, dtype=act)
+    idx = torch.stack([torch.randperm(S, device=dev)[:n_active] for _ in range(B)]).to(torch.int32).contiguous()
+    w0 = m.weights[0]
+    partial = torch.rand(B, H, S, device=dev)
+    scores = torch.rand(B, S, device=dev)
+    mask = torch.empty(B * S, dtype=torch.uint8, device=dev)
+    k = int(np.floor(cfg.ratio * S + 0.5))
+    refresh = torch.empty(B, max(k, 1), dtype=torch.int32, device=dev)
+    new = idx[:, :4].contiguous()
+
+    def timed_us(fn, reps=24):
+        for i in range(3):
+            fn(i)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(reps):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps * 1e3
+
+    rows = []
+
+    def add(name, bound, amount, us):
+        unit = "TFLOP/s" if bound == "tensor" else "GB/s"
+        peak = peaks["bf16_tflops_sustained"] if bound == "tensor" else peaks["hbm_gbs"]
+        ach = amount / (us * 1e-6) / (1e12 if bound == "tensor" else 1e9)
+        rows.append({"kernel": name, "bound": bound, "us": us, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak})
+
+    add("gather_layernorm (M x D)", "hbm", M * D * (4 + eb),
+        timed_us(lambda i: m.gather_layernorm(xs[i % rot].view(B, n_active, D), None, n_active, w0["ln2_g"], w0["ln2_b"], None, us[i % rot])))
+    add("scatter_kv", "hbm", 4.0 * M * D * eb,
+        timed_us(lambda i: m.scatter_kv(qkvs[i % rot][:, D:], qkvs[i % rot][:, 2 * D:], 3 * D, idx, n_active, caches[i % rot])))
+    add("attention (plain)", "hbm", 2.0 * B * S * D * eb + 2.0 * M * D * eb,
+        timed_us(lambda i: m.attention(qkvs[i % rot], 3 * D, n_active, caches[i % rot], None, None, o)))
+    for name, a_in, wname, bname, epi, out, N, K in (
+            ("gemm qkv", us[0], "w_qkv", "b_qkv", 0, qkvs[0], 3 * D, D), ("gemm out-proj (+residual)", o, "w_o", "b_o", 1, xs[0], D, D),
+            ("gemm fc1 (+GELU)", us[0], "w_fc1", "b_fc1", 2, g, F, D), ("gemm fc2 (+residual)", g, "w_fc2", "b_fc2", 1, xs[0], D, F)):
+        add("%s %dx%dx%d" % (name, M, N, K), "tensor", 2.0 * M * N * K,
+            timed_us(lambda i: m.linear(a_in, w0[wname], w0[bname], epi, out)))
+    add("topk (select_refresh, k=%d)" % k, "hbm", B * S * 5 + B * k * 4,
+        timed_us(lambda i: m.select_refresh(scores, new, None, k, refresh, mask)))
+    return rows
 
 
 def run_microbench(args):
