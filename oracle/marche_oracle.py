@@ -38,6 +38,14 @@ What is written out, and from where in the paper:
                            attention up to the scoring block, selection there, cache-aware
                            blocks after it; `generate_in_step` adds the fixed active budget
                            and the periodic full refresh of Section 4.3.
+* `mar_encoder`, `mar_decoder_input`, `mar_step`, `generate_mar`
+                           the two-stage shape of Section 3: Eq. 1 (encoder blocks on the known
+                           tokens only, nothing cached) and Eq. 2 (decoder over the whole sequence,
+                           mask embedding at masked positions), with the decoder scheduled as in
+                           Section 4.2 / 4.3.  Pinned by: encoder == full pass over the compacted
+                           sequence, masked rows never read, closed forms of the decoder input,
+                           decoder == the pinned uniform-stack functions on the same input,
+                           refresh-everything == full decoder.
 
 Readings where the paper is silent (block internals, tie rule, refresh ratio)
 are listed in the repository's design notes; each is marked "reading" below.
@@ -415,4 +423,123 @@ def generate(blocks, hidden0: np.ndarray, new_sets: List[np.ndarray], replacemen
         for b in range(B):
             hidden[b, G[b]] = rows[b]
         R = R_next
+    return log, cache
+
+
+# --------------------------------------------------------------------------
+# MAR's two-stage shape (Section 3, Eq. 1 and Eq. 2): an encoder over the known
+# tokens only, then a decoder over the whole sequence with mask embeddings.
+# --------------------------------------------------------------------------
+
+def mar_encoder(blocks: Sequence[Block], tokens_b: np.ndarray, known: np.ndarray, *, n_heads: int,
+                ln_eps: float) -> np.ndarray:
+    """Eq. 1 for one sample: the encoder blocks on the rows `known` of tokens_b [S][D] alone.
+    Keys and values are those of the known tokens of this very step; nothing is cached
+    (reading: the paper speaks of cached projections only for decoder layers).
+    Returns the encoder output rows [n_known][D] before the encoder's final norm."""
+    X = tokens_b[known]
+    n = len(known)
+    own = np.arange(n, dtype=np.int64)
+    for blk in blocks:
+        K_l = np.zeros((n, X.shape[1]), dtype=X.dtype)
+        V_l = np.zeros_like(K_l)
+        X, _ = _block(X, blk, K_l, V_l, own, n_heads, ln_eps, None)
+    return X
+
+
+def mar_decoder_input(h_enc: np.ndarray, known: np.ndarray, S: int, mar: Dict[str, np.ndarray],
+                      ln_eps: float) -> np.ndarray:
+    """The decoder's input of Eq. 2 for one sample, [S][D]: at a known position the encoder
+    output, normalised and projected to the decoder (reading: MAR's final encoder norm and its
+    encoder-to-decoder linear map), at a masked position the learned mask embedding; the
+    decoder's positional embedding is added to every position."""
+    X = np.tile(mar["mask_token"], (S, 1))
+    X[known] = linear(layer_norm(h_enc, mar["enc_norm_g"], mar["enc_norm_b"], ln_eps),
+                      mar["w_dec_embed"], mar["b_dec_embed"])
+    return X + mar["dec_pos"]
+
+
+def mar_step(blocks: Sequence[Block], mar: Dict[str, np.ndarray], tokens: np.ndarray, known_idx: np.ndarray,
+             cache: KVCache, new_idx: np.ndarray, prev_idx: Optional[np.ndarray], n_refresh: int,
+             z_out: np.ndarray, *, n_heads: int, n_enc: int, score_layer: int, full_decoder: bool,
+             ln_eps: float = 1e-6, real=np.float64, forced_refresh: Optional[np.ndarray] = None):
+    """One decoding step of the two-stage model (Eq. 1, Eq. 2) with the cache-aware decoder.
+
+    blocks[:n_enc] are the encoder, blocks[n_enc:] the decoder; cache rows of the encoder
+    blocks are not used.  tokens [B][S][D] holds the embedded known tokens (rows outside
+    known_idx are ignored); known_idx int32 [B][n_known] ascending.
+    full_decoder: every decoder block on every token (first step, periodic full refresh of
+    Section 4.3).  Otherwise the schedule of Section 4.2: decoder blocks up to score_layer on
+    every token, top-n_refresh selection there with G and N excluded, A = G u N u R afterwards.
+    Rows A (all rows when full_decoder) of z_out [B][S][D] receive the decoder output after
+    the decoder's final norm.
+    Returns (scores fp32 [B][S], refresh_idx int32 [B][n_refresh], active_idx int32 [B][nA])."""
+    B, S, D = tokens.shape
+    L = len(blocks)
+    if not (n_enc <= score_layer < L):
+        raise ValueError("score_layer must be a decoder block")
+    if not full_decoder and (not cache.filled or score_layer >= L - 1):
+        raise RuntimeError("cache-aware decoder needs a filled cache and a block after score_layer")
+    blocks = [{k: np.asarray(v, dtype=real) for k, v in blk.items()} for blk in blocks]
+    mar = {k: np.asarray(v, dtype=real) for k, v in mar.items()}
+    all_idx = np.arange(S, dtype=np.int64)
+    last_full = L - 1 if full_decoder else score_layer
+    scores = np.zeros((B, S), dtype=real)
+    X_full = []
+    for b in range(B):
+        known = np.asarray(known_idx[b], dtype=np.int64)
+        h_enc = mar_encoder(blocks[:n_enc], tokens[b].astype(real), known, n_heads=n_heads, ln_eps=ln_eps)
+        X = mar_decoder_input(h_enc, known, S, mar, ln_eps)
+        new = set(np.asarray(new_idx[b]).tolist())
+        scoring_rows = np.array([t in new for t in range(S)], dtype=bool)
+        for l in range(n_enc, last_full + 1):
+            X, sc = _block(X, blocks[l], cache.K[l, b], cache.V[l, b], all_idx, n_heads, ln_eps,
+                           scoring_rows if l == score_layer else None)
+            if sc is not None:
+                scores[b] = sc
+        X_full.append(X)
+    scores32 = scores.astype(np.float32)
+    refresh = select_refresh(scores32, new_idx, prev_idx, n_refresh)
+    if full_decoder:
+        cache.filled = True
+        A = np.tile(np.arange(S, dtype=np.int32), (B, 1))
+        for b in range(B):
+            z_out[b] = layer_norm(X_full[b], mar["dec_norm_g"], mar["dec_norm_b"], ln_eps).astype(z_out.dtype)
+        return scores32, refresh, A
+    R = refresh if forced_refresh is None else np.asarray(forced_refresh, dtype=np.int32)
+    A = active_set(new_idx, prev_idx, R)
+    for b in range(B):
+        idx = A[b].astype(np.int64)
+        X = X_full[b][idx]
+        for l in range(score_layer + 1, L):
+            X, _ = _block(X, blocks[l], cache.K[l, b], cache.V[l, b], idx, n_heads, ln_eps, None)
+        z_out[b, idx] = layer_norm(X, mar["dec_norm_g"], mar["dec_norm_b"], ln_eps).astype(z_out.dtype)
+    return scores32, refresh, A
+
+
+def generate_mar(blocks, mar, tokens0: np.ndarray, new_sets: List[np.ndarray], known_sets: List[np.ndarray],
+                 replacement, *, n_heads: int, n_enc: int, score_layer: int, budget: int = 64, period: int = 3,
+                 ln_eps: float = 1e-6, real=np.float64):
+    """A whole generation of the two-stage model under the schedule of Section 4.3: the decoder is
+    fully refreshed at the first and at every `period`-th step, otherwise it runs the in-step
+    selection with the fixed active budget K = budget - #G - #N.  After step t, rows G(t) of the
+    token embeddings are overwritten by replacement(t, #G(t)) and count as known from then on."""
+    B, S, D = tokens0.shape
+    tokens = tokens0.copy()
+    z = np.zeros_like(tokens0)
+    cache = KVCache(len(blocks), B, S, D, real=real)
+    empty = np.zeros((B, 0), dtype=np.int32)
+    log = []
+    for t, G in enumerate(new_sets):
+        N = new_sets[t - 1] if t > 0 else empty
+        full = t % period == 0
+        k = 0 if full else min(fixed_budget_refresh_count(budget, G.shape[1], N.shape[1]),
+                               S - G.shape[1] - N.shape[1])
+        scores, R, A = mar_step(blocks, mar, tokens, known_sets[t], cache, G, N, k, z, n_heads=n_heads,
+                                n_enc=n_enc, score_layer=score_layer, full_decoder=full, ln_eps=ln_eps, real=real)
+        log.append(dict(t=t, kind="full" if full else "in_step", active=A, new=G, prev=N, scores=scores,
+                        refresh=R, z=z.copy()))
+        rows = replacement(t, G.shape[1])
+        for b in range(B):
+            tokens[b, G[b]] = rows[b]
     return log, cache

@@ -17,4 +17,7 @@ from .workload import (  # noqa: F401
     replacement_rows,
     round_to_bf16,
     peaked_weights,
+    MAR_FIELDS,
+    make_mar_weights,
+    known_token_sets,
 )

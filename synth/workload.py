@@ -202,3 +202,45 @@ def replacement_rows(cfg: MarConfig, t: int, n_rows: int, seed: int = SEED_ROWS,
     rng = np.random.Generator(np.random.Philox(key=seed, counter=[t, 0, 0, 0]))
     B = cfg.B if batch is None else batch
     return rng.standard_normal((B, n_rows, cfg.D), dtype=np.float32)
+
+
+SEED_MAR = 4321
+MAR_FIELDS = ("enc_norm_g", "enc_norm_b", "w_dec_embed", "b_dec_embed", "mask_token", "dec_pos",
+              "dec_norm_g", "dec_norm_b")
+
+
+def make_mar_weights(cfg: MarConfig, seed: int = SEED_MAR) -> Dict[str, np.ndarray]:
+    """fp32 arrays of the two-stage model's glue: final encoder norm, encoder-to-decoder linear map
+    ([out][in]), mask embedding [D], decoder positional embedding [S][D], final decoder norm.
+    Norm gains 1 + N(0, 0.02^2); the embeddings N(0, 1) and N(0, 0.02^2) like the rest; for bf16
+    configs the matrix holds values exact in bf16 and fp16."""
+    rng = np.random.Generator(np.random.Philox(seed))
+    D, S = cfg.D, cfg.S
+    shapes = {"enc_norm_g": (D,), "enc_norm_b": (D,), "w_dec_embed": (D, D), "b_dec_embed": (D,),
+              "mask_token": (D,), "dec_pos": (S, D), "dec_norm_g": (D,), "dec_norm_b": (D,)}
+    out = {}
+    for name in MAR_FIELDS:
+        a = rng.standard_normal(shapes[name], dtype=np.float32)
+        if name not in ("mask_token", "dec_pos"):
+            a = a * np.float32(0.02)
+        if name.endswith("_g"):
+            a = a + np.float32(1.0)
+        if name == "w_dec_embed":
+            # one-over-sqrt(D) scale keeps the projected rows at unit size like the mask embedding
+            a = a * np.float32(50.0 / math.sqrt(D))
+            if cfg.dtype == "bf16":
+                a = round_to_bf16(a).astype(np.float16).astype(np.float32)
+        out[name] = np.ascontiguousarray(a, dtype=np.float32)
+    return out
+
+
+def known_token_sets(cfg: MarConfig, new_sets: List[np.ndarray]) -> List[np.ndarray]:
+    """List over steps t of int32 [B][n_known(t)], ascending: the buffer positions plus every
+    position generated before step t (the tokens that are not masked at step t)."""
+    B = new_sets[0].shape[0]
+    known = np.tile(np.arange(cfg.n_buffer, dtype=np.int32), (B, 1))
+    out = []
+    for G in new_sets:
+        out.append(np.ascontiguousarray(np.sort(known, axis=1)))
+        known = np.concatenate([known, G.astype(np.int32)], axis=1)
+    return out
