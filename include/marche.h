@@ -200,6 +200,57 @@ int marche_step_in_step_selection(marche_ctx* ctx, const float* hidden, void* kv
                                   int32_t* refresh_idx, int32_t* active_idx,
                                   void* workspace, size_t workspace_bytes, marche_stream stream);
 
+/* ---------------------------------------------------------------- two-stage model (Section 3) */
+
+/* Glue of MAR's encoder/decoder shape around the L blocks; all device pointers, borrowed like the
+ * block weights.  Reading: the encoder output passes a final LayerNorm and a linear map into the
+ * decoder width (equal to D here), the decoder adds its own learned positional embedding to every
+ * position and ends in a final LayerNorm. */
+typedef struct {
+  const float* enc_norm_g;  const float* enc_norm_b;   /* [D]   final encoder norm                 */
+  const void* w_dec_embed;  const float* b_dec_embed;  /* A [D][D] ([out][in]), float [D]          */
+  const float* mask_token;                             /* [D]   embedding of a masked position     */
+  const float* dec_pos;                                /* [S][D] decoder positional embedding      */
+  const float* dec_norm_g;  const float* dec_norm_b;   /* [D]   final decoder norm                 */
+} marche_mar_weights;
+
+/* Registers the glue weights; needs 1 <= n_enc_blocks < n_blocks (MARCHE_EINVAL otherwise, also
+ * for a NULL member).  Nothing is enqueued. */
+int marche_set_mar_weights(marche_ctx* ctx, const marche_mar_weights* w);
+
+/* One decoding step of the two-stage model.
+ *   Eq. 1   blocks 0 .. E-1 (E = n_enc_blocks) run on the known tokens only: rows known_idx of
+ *           `tokens` are gathered, attend to one another and to nothing else.  These blocks are
+ *           recomputed in every step and cache nothing across steps (the paper keeps cached
+ *           projections only in decoder layers); their slices of kv_cache serve as per-step
+ *           scratch in a compact [2][B][n_known][D] layout.
+ *   Eq. 2   the decoder's input is, at a known position, w_dec_embed * LN_enc(encoder row) +
+ *           b_dec_embed, at every other position mask_token; dec_pos is added everywhere.
+ *   decoder blocks E .. L-1.  full_decoder != 0: on every token (the first step and the periodic
+ *           full refresh of Section 4.3); all S rows of z_out are written; marks kv_cache filled.
+ *           full_decoder == 0: the schedule of Section 4.2 - blocks E .. score_layer on every
+ *           token, the n_refresh best-scoring tokens outside new_idx u prev_idx selected there,
+ *           the later blocks cache-aware on A = new | prev | refresh (Algorithm 1); rows A of
+ *           z_out are written, other rows keep their bytes.
+ *   z_out   device float [B][S][D]: decoder output after the final decoder norm (the vectors the
+ *           sampler of Eq. 3 is conditioned on).
+ *   tokens  device float [B][S][D]: embedded input tokens; rows outside known_idx are never read.
+ *   known_idx  device int32 [B][n_known], ascending within a sample; 1 <= n_known <= S.
+ *   new_idx / prev_idx / forced_refresh / refresh_idx / active_idx: as for
+ *           marche_step_in_step_selection; refresh_idx may be NULL when n_refresh == 0 and
+ *           active_idx may be NULL when full_decoder != 0.  The relevance scores of block
+ *           score_layer are computed in both modes (marche_get_scores).
+ *   workspace  marche_workspace_bytes(ctx, S).
+ * Needs marche_set_mar_weights, E <= score_layer, and for full_decoder == 0 score_layer < L-1
+ * (MARCHE_EINVAL) and a filled cache (MARCHE_ECACHE).  A cache driven by this call holds encoder
+ * scratch in its first E slices: run marche_full_step before using it with the uniform-stack calls. */
+int marche_mar_step(marche_ctx* ctx, int full_decoder, const float* tokens,
+                    const int32_t* known_idx, int n_known, void* kv_cache,
+                    const int32_t* new_idx, int n_new, const int32_t* prev_idx, int n_prev,
+                    int n_refresh, const int32_t* forced_refresh, float* z_out,
+                    int32_t* refresh_idx, int32_t* active_idx,
+                    void* workspace, size_t workspace_bytes, marche_stream stream);
+
 /* Top-K refresh selection alone (Section 4.2, "select the top-K tokens with the
  * highest relevance scores"): scores device float [B][S] (finite); candidates
  * are all tokens outside new_idx and exclude_idx; writes refresh_idx device

@@ -34,6 +34,14 @@ class MarcheBlockWeights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in BLOCK_FIELDS]
 
 
+MAR_FIELDS = ("enc_norm_g", "enc_norm_b", "w_dec_embed", "b_dec_embed", "mask_token", "dec_pos",
+              "dec_norm_g", "dec_norm_b")
+
+
+class MarcheMarWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in MAR_FIELDS]
+
+
 class MarcheError(RuntimeError):
     def __init__(self, code: int, detail: str = ""):
         self.code = code
@@ -50,6 +58,8 @@ _SIGNATURES = {
     "marche_step": (C.c_int, [_vp, _vp, _vp, _vp, _i, _vp, _i, _vp, _i, _f, _vp, _vp, C.POINTER(C.c_int), _vp, _sz, _vp]),
     "marche_full_step": (C.c_int, [_vp, _vp, _vp, _vp, _i, _vp, _i, _f, _vp, _vp, C.POINTER(C.c_int), _vp, _sz, _vp]),
     "marche_step_in_step_selection": (C.c_int, [_vp, _vp, _vp, _vp, _i, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "marche_set_mar_weights": (C.c_int, [_vp, C.POINTER(MarcheMarWeights)]),
+    "marche_mar_step": (C.c_int, [_vp, _i, _vp, _vp, _i, _vp, _vp, _i, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "marche_select_refresh": (C.c_int, [_vp, _vp, _vp, _i, _vp, _i, _i, _vp, _vp, _vp]),
     "marche_select_refresh_policy": (C.c_int, [_vp, _vp, _vp, _i, _vp, _i, _i, _i, C.c_uint32, _vp, _vp, _vp]),
     "marche_select_refresh_static": (C.c_int, [_vp, _vp, _vp, _i, _vp, _i, _i, _vp, _vp]),
@@ -120,6 +130,14 @@ def upload_weights(blocks: Sequence[Dict], dtype: str, device="cuda") -> List[Di
             d[name] = t.to(device=device, dtype=mt if name in MATRIX_FIELDS else torch.float32).contiguous()
         out.append(d)
     return out
+
+
+def upload_mar_weights(mar: Dict, dtype: str, device="cuda") -> Dict[str, torch.Tensor]:
+    """Copies the two-stage model's glue parameters to the device (the encoder-to-decoder matrix
+    as a projection operand, everything else fp32)."""
+    mt = torch.float16 if dtype == "bf16" else torch.float32
+    return {name: torch.as_tensor(mar[name]).to(device=device, dtype=mt if name == "w_dec_embed" else torch.float32)
+            .contiguous() for name in MAR_FIELDS}
 
 
 class Marche:
@@ -216,6 +234,24 @@ class Marche:
             self.h, _ptr(hidden), _ptr(kv_cache), _ptr(new_idx), 0 if new_idx is None else new_idx.shape[1],
             _ptr(prev_idx), 0 if prev_idx is None else prev_idx.shape[1], n_refresh, _ptr(forced_refresh),
             _ptr(hidden_out), _ptr(refresh_idx), _ptr(active_idx), _ptr(workspace), workspace.numel(), _stream(stream)))
+
+    def set_mar_weights(self, mar: Dict[str, torch.Tensor]):
+        w = MarcheMarWeights()
+        for name in MAR_FIELDS:
+            t = mar[name]
+            want = self.operand_dtype if name == "w_dec_embed" else torch.float32
+            assert t.is_cuda and t.is_contiguous() and t.dtype == want, name
+            setattr(w, name, t.data_ptr())
+        self.mar_weights = dict(mar)          # keeps the device tensors alive
+        self._check(self.lib.marche_set_mar_weights(self.h, C.byref(w)))
+
+    def mar_step(self, full_decoder, tokens, known_idx, kv_cache, new_idx, prev_idx, n_refresh, forced_refresh, z_out,
+                 refresh_idx, active_idx, workspace, stream=None):
+        self._check(self.lib.marche_mar_step(
+            self.h, 1 if full_decoder else 0, _ptr(tokens), _ptr(known_idx), known_idx.shape[1], _ptr(kv_cache),
+            _ptr(new_idx), 0 if new_idx is None else new_idx.shape[1],
+            _ptr(prev_idx), 0 if prev_idx is None else prev_idx.shape[1], n_refresh, _ptr(forced_refresh),
+            _ptr(z_out), _ptr(refresh_idx), _ptr(active_idx), _ptr(workspace), workspace.numel(), _stream(stream)))
 
     def select_refresh(self, scores, new_idx, exclude_idx, k, refresh_idx, mask_scratch, stream=None):
         self._check(self.lib.marche_select_refresh(

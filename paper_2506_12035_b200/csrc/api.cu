@@ -27,6 +27,8 @@ using namespace marche;
 struct marche_ctx {
   marche_config cfg;
   std::vector<marche_block_weights> blocks;
+  marche_mar_weights mar{};                           // glue of the two-stage model (marche_set_mar_weights)
+  bool has_mar = false;
   int device = 0;
   bool bf16 = false;
   size_t eb = 4;
@@ -56,7 +58,7 @@ namespace {
 inline size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 struct WsLayout {
-  size_t scores, partial, cand, is_new, turn, turn_bytes, x, x2, u, qkv, o, g, total;
+  size_t scores, partial, cand, is_new, turn, turn_bytes, x, x2, x3, u, qkv, o, g, total;
 };
 
 WsLayout ws_layout(const marche_ctx* c, int nA) {
@@ -72,6 +74,7 @@ WsLayout ws_layout(const marche_ctx* c, int nA) {
   w.turn = off;    off += align256(w.turn_bytes);
   w.x = off;       off += align256(M * D * sizeof(float));
   w.x2 = off;      off += align256(M * D * sizeof(float));   // second residual buffer (in-step selection)
+  w.x3 = off;      off += align256(M * D * sizeof(float));   // decoder input of the two-stage step
   w.u = off;       off += align256(M * D * eb);
   w.qkv = off;     off += align256(M * 3 * D * eb);
   w.o = off;       off += align256(M * D * eb);
@@ -128,8 +131,9 @@ int do_linear(marche_ctx* ctx, int cls, const void* a, int lda, int M, const voi
 }
 
 int do_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void* cache_layer, const uint8_t* is_new,
-                 float* partial, void* o, cudaStream_t st) {
+                 float* partial, void* o, cudaStream_t st, int S_kv = 0) {
   const marche_config& c = ctx->cfg;
+  const int S = S_kv > 0 ? S_kv : c.seq_len;            // tokens per sample in cache_layer [2][B][S][D]
   if (n > 0) mark(ctx, MARCHE_KC_ATTENTION, st);
   const bool tc = ctx->bf16 && !ctx->force_simt && (c.head_dim == 64 || c.head_dim == 80) && ld_q % 2 == 0 &&
                   ((uintptr_t)q & 3) == 0 && ((uintptr_t)cache_layer & 15) == 0;
@@ -142,20 +146,20 @@ int do_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void* ca
   const bool tc5 = tc && c.head_dim == 64 && ld_q % 8 == 0 && ((uintptr_t)q & 15) == 0 &&
                    (ctx->attn_tc == 1 || (ctx->attn_tc < 0 && n > tc_min));
   if (tc5)
-    MARCHE_TRY(launch_attention_tcgen05(q, ld_q, c.batch, n, c.seq_len, c.n_heads, c.head_dim, cache_layer, is_new,
+    MARCHE_TRY(launch_attention_tcgen05(q, ld_q, c.batch, n, S, c.n_heads, c.head_dim, cache_layer, is_new,
                                         partial, o, ctx->status_dev, st), "attention_tcgen05");
   else if (tc)
-    MARCHE_TRY(launch_attention_mma(q, ld_q, c.batch, n, c.seq_len, c.n_heads, c.head_dim, cache_layer, is_new,
+    MARCHE_TRY(launch_attention_mma(q, ld_q, c.batch, n, S, c.n_heads, c.head_dim, cache_layer, is_new,
                                     partial, o, ctx->status_dev, st), "attention_mma");
   else
-    MARCHE_TRY(launch_attention_simt(ctx->bf16, q, ld_q, c.batch, n, c.seq_len, c.n_heads, c.head_dim, cache_layer,
+    MARCHE_TRY(launch_attention_simt(ctx->bf16, q, ld_q, c.batch, n, S, c.n_heads, c.head_dim, cache_layer,
                                      is_new, partial, o, st), "attention");
   return MARCHE_OK;
 }
 
 struct StackBufs {
   float* scores; float* partial; uint8_t* cand; uint8_t* is_new;
-  float* x; float* x2; char* u; char* qkv; char* o; char* g;
+  float* x; float* x2; float* x3; char* u; char* qkv; char* o; char* g;
   int* turn;
 };
 
@@ -169,6 +173,7 @@ StackBufs carve(void* workspace, const WsLayout& w) {
   b.turn = (int*)(ws + w.turn);
   b.x = (float*)(ws + w.x);
   b.x2 = (float*)(ws + w.x2);
+  b.x3 = (float*)(ws + w.x3);
   b.u = ws + w.u;
   b.qkv = ws + w.qkv;
   b.o = ws + w.o;
@@ -180,13 +185,17 @@ StackBufs carve(void* workspace, const WsLayout& w) {
 // nA == S).  When gather_src is non-null the first block's LayerNorm gathers its rows from
 // gather_src[b][idx][:] (float [B][src_rows][D]) and writes the compact residual rows to x;
 // otherwise x already holds them.  is_new (flags of the scoring queries) is used at the scoring block.
+// S_kv > 0: these blocks keep only S_kv tokens per sample, laid out [2][B][S_kv][D] at the start of each
+// block's cache slice (the encoder over the known tokens, whose K/V do not outlive the step).
 int run_blocks(marche_ctx* ctx, int l_begin, int l_end, const float* gather_src, int src_rows, const int32_t* idx,
-               int nA, float* x, const StackBufs& bf, void* kv_cache, const uint8_t* is_new, cudaStream_t st) {
+               int nA, float* x, const StackBufs& bf, void* kv_cache, const uint8_t* is_new, cudaStream_t st,
+               int S_kv = 0) {
   const marche_config& c = ctx->cfg;
-  const int B = c.batch, S = c.seq_len, D = c.width, F = c.mlp_dim;
+  const int B = c.batch, S = S_kv > 0 ? S_kv : c.seq_len, D = c.width, F = c.mlp_dim;
   const int M = B * nA;
   const size_t eb = ctx->eb;
-  const size_t layer_bytes = (size_t)2 * B * S * D * eb;
+  const size_t layer_bytes = (size_t)2 * B * c.seq_len * D * eb;
+  const int32_t* kv_idx = S_kv > 0 ? nullptr : idx;   // compact layout: row j of the sample is token j
   for (int l = l_begin; l < l_end; ++l) {
     const marche_block_weights& bw = ctx->blocks[l];
     char* cache_l = (char*)kv_cache + (size_t)l * layer_bytes;
@@ -202,7 +211,7 @@ int run_blocks(marche_ctx* ctx, int l_begin, int l_end, const float* gather_src,
     if (ctx->attn_mode == 1 && ctx->bf16 && !ctx->force_simt) {
       // two-segment attention: fresh K/V read in place, cache write-back by the same kernel
       mark(ctx, MARCHE_KC_ATTENTION, st);
-      MARCHE_TRY(launch_attention_twoseg(bf.qkv, 3 * D, D, 2 * D, B, nA, S, c.n_heads, c.head_dim, idx, cache_l,
+      MARCHE_TRY(launch_attention_twoseg(bf.qkv, 3 * D, D, 2 * D, B, nA, S, c.n_heads, c.head_dim, kv_idx, cache_l,
                                          l == ctx->score_layer ? is_new : nullptr, bf.partial, bf.o, ctx->status_dev, st),
                  "attention_twoseg");
     } else if (ctx->fuse_writeback && ctx->bf16 && !ctx->force_simt && ctx->attn_tc != 1 &&
@@ -212,12 +221,13 @@ int run_blocks(marche_ctx* ctx, int l_begin, int l_end, const float* gather_src,
       mark(ctx, MARCHE_KC_ATTENTION, st);
       MARCHE_TRY(launch_attention_mma(bf.qkv, 3 * D, B, nA, S, c.n_heads, c.head_dim, cache_l,
                                       l == ctx->score_layer ? is_new : nullptr, bf.partial, bf.o, ctx->status_dev, st,
-                                      true, idx, D, 2 * D), "attention_mma_wb");
+                                      true, kv_idx, D, 2 * D), "attention_mma_wb");
     } else {
       mark(ctx, MARCHE_KC_SCATTER_KV, st);
-      MARCHE_TRY(launch_scatter_kv(ctx->bf16, bf.qkv + (size_t)D * eb, bf.qkv + (size_t)2 * D * eb, 3 * D, idx, B, nA,
+      MARCHE_TRY(launch_scatter_kv(ctx->bf16, bf.qkv + (size_t)D * eb, bf.qkv + (size_t)2 * D * eb, 3 * D, kv_idx, B, nA,
                                    S, D, cache_l, st), "scatter_kv");
-      rc = do_attention(ctx, bf.qkv, 3 * D, nA, cache_l, l == ctx->score_layer ? is_new : nullptr, bf.partial, bf.o, st);
+      rc = do_attention(ctx, bf.qkv, 3 * D, nA, cache_l, l == ctx->score_layer ? is_new : nullptr, bf.partial, bf.o, st,
+                        S);
       if (rc) return rc;
     }
     rc = do_linear(ctx, MARCHE_KC_GEMM_O, bf.o, D, M, bw.w_o, bw.b_o, D, D, MARCHE_EPI_BIAS_RESIDUAL, x, st, bf.turn);
@@ -297,6 +307,75 @@ int run_in_step(marche_ctx* ctx, const float* hidden, void* kv_cache, const int3
   if (rc) return rc;
   mark(ctx, MARCHE_KC_SCATTER_ROWS, st);
   MARCHE_TRY(launch_scatter_rows(bf.x2, active_idx, B, nA, S, D, hidden_out, st), "scatter_rows");
+  return MARCHE_OK;
+}
+
+// One step of the two-stage model: encoder blocks [0, E) on the known tokens only (Eq. 1), the
+// decoder's input assembled from the projected encoder rows and the mask embedding (Eq. 2), then
+// the decoder blocks [E, L) either on every token or under the in-step selection schedule.
+int run_mar(marche_ctx* ctx, bool full_decoder, const float* tokens, const int32_t* known_idx, int n_known,
+            void* kv_cache, const int32_t* new_idx, int n_new, const int32_t* prev_idx, int n_prev, int k,
+            const int32_t* forced_refresh, float* z_out, int32_t* refresh_idx, int32_t* active_idx, void* workspace,
+            size_t ws_bytes, cudaStream_t st) {
+  const marche_config& c = ctx->cfg;
+  const int B = c.batch, S = c.seq_len, D = c.width, H = c.n_heads, L = c.n_blocks, E = c.n_enc_blocks;
+  const int sl = ctx->score_layer;
+  if (!ctx->has_mar) return MARCHE_EINVAL;
+  if (!tokens || !known_idx || !kv_cache || !z_out || !workspace || tokens == z_out) return MARCHE_EINVAL;
+  if (E < 1 || E >= L || sl < E) return MARCHE_EINVAL;
+  if (n_known < 1 || n_known > S || n_new < 0 || n_prev < 0 || k < 0 || n_new + n_prev + k > S) return MARCHE_EINVAL;
+  if ((n_new > 0 && !new_idx) || (n_prev > 0 && !prev_idx) || (k > 0 && !refresh_idx)) return MARCHE_EINVAL;
+  const int nA = n_new + n_prev + k;
+  if (!full_decoder && (sl >= L - 1 || nA < 1 || !active_idx)) return MARCHE_EINVAL;
+  if (((uintptr_t)workspace & 255) != 0) return MARCHE_EINVAL;
+  const WsLayout w = ws_layout(ctx, S);
+  if (ws_bytes < w.total) return MARCHE_EWORKSPACE;
+  const StackBufs bf = carve(workspace, w);
+  const marche_mar_weights& mw = ctx->mar;
+  if (ctx->bf16 && ctx->stream_k) MARCHE_TRY(cudaMemsetAsync(bf.turn, 0, w.turn_bytes, st), "memset");
+
+  mark(ctx, MARCHE_KC_FLAGS, st);
+  MARCHE_TRY(launch_step_flags(nullptr, S, new_idx, n_new, prev_idx, n_prev, B, S, bf.is_new, bf.cand, st), "flags");
+  // ---- Eq. 1: encoder on the compacted known tokens; its K/V live only inside this step
+  int rc = run_blocks(ctx, 0, E, tokens, S, known_idx, n_known, bf.x, bf, kv_cache, nullptr, st, n_known);
+  if (rc) return rc;
+  // ---- Eq. 2: x3[b][s] = mask + pos[s];  x3[b][known] = W_de * LN(h_enc) + b_de + pos[known]
+  mark(ctx, MARCHE_KC_GATHER_LN, st);
+  MARCHE_TRY(launch_gather_layernorm(ctx->bf16, bf.x, n_known, nullptr, B, n_known, D, mw.enc_norm_g, mw.enc_norm_b,
+                                     ctx->eps, nullptr, bf.u, st), "encoder_norm");
+  mark(ctx, MARCHE_KC_OTHER, st);
+  MARCHE_TRY(launch_gather_table_rows(mw.dec_pos, known_idx, (long)B * n_known, D, bf.x2, st), "gather_table_rows");
+  rc = do_linear(ctx, MARCHE_KC_OTHER, bf.u, D, B * n_known, mw.w_dec_embed, mw.b_dec_embed, D, D,
+                 MARCHE_EPI_BIAS_RESIDUAL, bf.x2, st, bf.turn);
+  if (rc) return rc;
+  mark(ctx, MARCHE_KC_OTHER, st);
+  MARCHE_TRY(launch_fill_mask_rows(mw.mask_token, mw.dec_pos, B, S, D, bf.x3, st), "fill_mask_rows");
+  mark(ctx, MARCHE_KC_SCATTER_ROWS, st);
+  MARCHE_TRY(launch_scatter_rows(bf.x2, known_idx, B, n_known, S, D, bf.x3, st), "scatter_rows");
+
+  // ---- decoder
+  if (full_decoder) {
+    rc = run_blocks(ctx, E, L, bf.x3, S, nullptr, S, bf.x, bf, kv_cache, bf.is_new, st);
+    if (rc) return rc;
+    mark(ctx, MARCHE_KC_TOPK, st);
+    MARCHE_TRY(launch_topk(bf.partial, H, bf.scores, bf.cand, B, S, k, refresh_idx, st), "topk");
+    mark(ctx, MARCHE_KC_GATHER_LN, st);
+    MARCHE_TRY(launch_gather_layernorm(false, bf.x, S, nullptr, B, S, D, mw.dec_norm_g, mw.dec_norm_b, ctx->eps,
+                                       nullptr, z_out, st), "decoder_norm");
+    return MARCHE_OK;
+  }
+  rc = run_blocks(ctx, E, sl + 1, bf.x3, S, nullptr, S, bf.x, bf, kv_cache, bf.is_new, st);
+  if (rc) return rc;
+  mark(ctx, MARCHE_KC_TOPK, st);
+  MARCHE_TRY(launch_topk(bf.partial, H, bf.scores, bf.cand, B, S, k, refresh_idx, st), "topk");
+  mark(ctx, MARCHE_KC_OTHER, st);
+  MARCHE_TRY(launch_build_active(new_idx, n_new, prev_idx, n_prev, forced_refresh ? forced_refresh : refresh_idx, k, B,
+                                 active_idx, st), "build_active");
+  rc = run_blocks(ctx, sl + 1, L, bf.x, S, active_idx, nA, bf.x2, bf, kv_cache, nullptr, st);
+  if (rc) return rc;
+  mark(ctx, MARCHE_KC_GATHER_LN, st);
+  MARCHE_TRY(launch_gather_layernorm(false, bf.x2, nA, nullptr, B, nA, D, mw.dec_norm_g, mw.dec_norm_b, ctx->eps,
+                                     nullptr, z_out, st, active_idx, S), "decoder_norm");
   return MARCHE_OK;
 }
 
@@ -423,6 +502,34 @@ int marche_step_in_step_selection(marche_ctx* ctx, const float* hidden, void* kv
   if (!e || !e->second) return MARCHE_ECACHE;
   return run_in_step(ctx, hidden, kv_cache, new_idx, n_new, prev_idx, n_prev, n_refresh, forced_refresh, hidden_out,
                      refresh_idx, active_idx, workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+int marche_set_mar_weights(marche_ctx* ctx, const marche_mar_weights* w) {
+  if (!ctx || !w) return MARCHE_EINVAL;
+  if (!w->enc_norm_g || !w->enc_norm_b || !w->w_dec_embed || !w->b_dec_embed || !w->mask_token || !w->dec_pos ||
+      !w->dec_norm_g || !w->dec_norm_b)
+    return MARCHE_EINVAL;
+  if (ctx->cfg.n_enc_blocks < 1 || ctx->cfg.n_enc_blocks >= ctx->cfg.n_blocks) return MARCHE_EINVAL;
+  ctx->mar = *w;
+  ctx->has_mar = true;
+  return MARCHE_OK;
+}
+
+int marche_mar_step(marche_ctx* ctx, int full_decoder, const float* tokens, const int32_t* known_idx, int n_known,
+                    void* kv_cache, const int32_t* new_idx, int n_new, const int32_t* prev_idx, int n_prev,
+                    int n_refresh, const int32_t* forced_refresh, float* z_out, int32_t* refresh_idx,
+                    int32_t* active_idx, void* workspace, size_t workspace_bytes, marche_stream stream) {
+  if (!ctx) return MARCHE_EINVAL;
+  auto* e = find_cache(ctx, kv_cache);
+  if (!full_decoder && (!e || !e->second)) return MARCHE_ECACHE;
+  const int rc = run_mar(ctx, full_decoder != 0, tokens, known_idx, n_known, kv_cache, new_idx, n_new, prev_idx, n_prev,
+                         n_refresh, forced_refresh, z_out, refresh_idx, active_idx, workspace, workspace_bytes,
+                         (cudaStream_t)stream);
+  if (rc == MARCHE_OK && full_decoder) {
+    if (e) e->second = true;
+    else ctx->caches.emplace_back(kv_cache, true);
+  }
+  return rc;
 }
 
 int marche_select_refresh(marche_ctx* ctx, const float* scores, const int32_t* new_idx, int n_new,

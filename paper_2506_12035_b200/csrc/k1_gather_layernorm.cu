@@ -18,7 +18,7 @@ __global__ void __launch_bounds__(kLnWarps * 32)
 gather_layernorm_kernel(const float* __restrict__ src, int src_rows, const int32_t* __restrict__ idx,
                         int n, int total_rows, const float* __restrict__ gamma,
                         const float* __restrict__ beta, float eps, float* __restrict__ x_out,
-                        TOut* __restrict__ u_out) {
+                        TOut* __restrict__ u_out, const int32_t* __restrict__ out_idx, int out_rows) {
   constexpr int D = NV * 128;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long r = (long)blockIdx.x * kLnWarps + warp;
@@ -51,7 +51,9 @@ gather_layernorm_kernel(const float* __restrict__ src, int src_rows, const int32
   }
   const float4* g4 = reinterpret_cast<const float4*>(gamma);
   const float4* b4 = reinterpret_cast<const float4*>(beta);
-  TOut* uo = u_out + r * D;
+  // out_rows > 0: the normalised row goes to row out_idx[r] (identity when NULL) of a [B][out_rows][D] array
+  const long orow = out_rows > 0 ? (long)b * out_rows + (out_idx ? out_idx[r] : j) : r;
+  TOut* uo = u_out + orow * D;
 #pragma unroll
   for (int i = 0; i < NV; ++i) {
     const float4 g = __ldg(g4 + i * 32 + lane), be = __ldg(b4 + i * 32 + lane);
@@ -64,7 +66,7 @@ gather_layernorm_kernel(const float* __restrict__ src, int src_rows, const int32
 template <typename TOut>
 static cudaError_t launch_ln_t(const float* src, int src_rows, const int32_t* idx, int B, int n, int D,
                                const float* gamma, const float* beta, float eps, float* x_out, TOut* u_out,
-                               cudaStream_t st) {
+                               cudaStream_t st, const int32_t* out_idx, int out_rows) {
   const long rows = (long)B * n;
   if (rows == 0) return cudaSuccess;
   const unsigned grid = (unsigned)((rows + kLnWarps - 1) / kLnWarps);
@@ -72,7 +74,7 @@ static cudaError_t launch_ln_t(const float* src, int src_rows, const int32_t* id
 #define MARCHE_LN_CASE(NV_)                                                                          \
   case NV_:                                                                                          \
     err = launch_pdl(gather_layernorm_kernel<TOut, NV_>, dim3(grid), dim3(kLnWarps * 32), 0, st, src, src_rows, \
-                     idx, n, (int)rows, gamma, beta, eps, x_out, u_out);                             \
+                     idx, n, (int)rows, gamma, beta, eps, x_out, u_out, out_idx, out_rows);          \
     break;
   switch (D / 128) {
     MARCHE_LN_CASE(1) MARCHE_LN_CASE(2) MARCHE_LN_CASE(3) MARCHE_LN_CASE(4) MARCHE_LN_CASE(5)
@@ -87,11 +89,12 @@ static cudaError_t launch_ln_t(const float* src, int src_rows, const int32_t* id
 
 cudaError_t launch_gather_layernorm(bool half_out, const float* src, int src_rows, const int32_t* idx,
                                     int B, int n, int D, const float* gamma, const float* beta, float eps,
-                                    float* x_out, void* u_out, cudaStream_t st) {
+                                    float* x_out, void* u_out, cudaStream_t st, const int32_t* out_idx,
+                                    int out_rows) {
   if (D % 128 != 0) return cudaErrorInvalidValue;
   if (half_out)
-    return launch_ln_t<f16>(src, src_rows, idx, B, n, D, gamma, beta, eps, x_out, (f16*)u_out, st);
-  return launch_ln_t<float>(src, src_rows, idx, B, n, D, gamma, beta, eps, x_out, (float*)u_out, st);
+    return launch_ln_t<f16>(src, src_rows, idx, B, n, D, gamma, beta, eps, x_out, (f16*)u_out, st, out_idx, out_rows);
+  return launch_ln_t<float>(src, src_rows, idx, B, n, D, gamma, beta, eps, x_out, (float*)u_out, st, out_idx, out_rows);
 }
 
 }  // namespace marche

@@ -3,6 +3,7 @@
 //  * scatter_kv:   cache write-back of the active rows' fresh K, V (Algorithm 1 line 11).
 //  * scatter_rows: fp32 row scatter (hidden_out rows of the active tokens; sampled rows
 //                  into the stack input).
+//  * gather_table_rows, fill_mask_rows: assembly of the decoder's input (Eq. 2).
 //  * step_flags:   per-step bookkeeping of the token sets of Algorithm 1 lines 1-4:
 //                  which active rows are generating tokens, which tokens may be picked
 //                  for refresh.
@@ -58,6 +59,36 @@ gather_rows_kernel(const float4* __restrict__ src, const int32_t* __restrict__ i
   const float4* s = src + ((long)b * S + idx[r]) * row_vecs;
   float4* d = out + r * row_vecs;
   for (int c = lane; c < row_vecs; c += 32) d[c] = __ldg(s + c);
+}
+
+// out[r] = table[idx[r]]: rows of a table shared by all samples (positional embedding), one warp per row.
+__global__ void __launch_bounds__(256)
+gather_table_rows_kernel(const float4* __restrict__ table, const int32_t* __restrict__ idx, int row_vecs,
+                         long total_rows, float4* __restrict__ out) {
+  const long r = (long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (r >= total_rows) return;
+  pdl_sync();
+  const float4* s = table + (long)idx[r] * row_vecs;
+  float4* d = out + r * row_vecs;
+  for (int c = lane; c < row_vecs; c += 32) d[c] = __ldg(s + c);
+}
+
+// out[b][s] = mask_token + pos[s] for every token of every sample (Eq. 2: the decoder's input at a
+// masked position); the rows of known tokens are overwritten afterwards.
+__global__ void __launch_bounds__(256)
+fill_mask_rows_kernel(const float4* __restrict__ mask_token, const float4* __restrict__ pos, int S, int row_vecs,
+                      long total_rows, float4* __restrict__ out) {
+  const long r = (long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (r >= total_rows) return;
+  pdl_sync();
+  const float4* p = pos + (r % S) * row_vecs;
+  float4* d = out + r * row_vecs;
+  for (int c = lane; c < row_vecs; c += 32) {
+    const float4 m = __ldg(mask_token + c), q = __ldg(p + c);
+    d[c] = make_float4(m.x + q.x, m.y + q.y, m.z + q.z, m.w + q.w);
+  }
 }
 
 // One CTA per sample.  mark bit0 = generating token, bit1 = excluded token.
@@ -156,6 +187,22 @@ cudaError_t launch_gather_rows(const float* src, const int32_t* idx, int B, int 
   if (total == 0) return cudaSuccess;
   return launch_pdl(gather_rows_kernel, dim3((unsigned)((total + 7) / 8)), dim3(256), 0, st, (const float4*)src, idx, n,
                     S, D / 4, total, (float4*)out);
+}
+
+cudaError_t launch_gather_table_rows(const float* table, const int32_t* idx, long total_rows, int D, float* out,
+                                     cudaStream_t st) {
+  if (D % 4) return cudaErrorInvalidValue;
+  if (total_rows == 0) return cudaSuccess;
+  return launch_pdl(gather_table_rows_kernel, dim3((unsigned)((total_rows + 7) / 8)), dim3(256), 0, st,
+                    (const float4*)table, idx, D / 4, total_rows, (float4*)out);
+}
+
+cudaError_t launch_fill_mask_rows(const float* mask_token, const float* pos, int B, int S, int D, float* out,
+                                  cudaStream_t st) {
+  if (D % 4) return cudaErrorInvalidValue;
+  const long total = (long)B * S;
+  return launch_pdl(fill_mask_rows_kernel, dim3((unsigned)((total + 7) / 8)), dim3(256), 0, st,
+                    (const float4*)mask_token, (const float4*)pos, S, D / 4, total, (float4*)out);
 }
 
 cudaError_t launch_step_flags(const int32_t* active_idx, int n_active, const int32_t* new_idx, int n_new,

@@ -11,7 +11,8 @@ namespace marche {
 // K1: gather + LayerNorm (output fp16 when half_out, else fp32).  rows = B*n; src row of (b, j) is src[b][idx ? idx[b][j] : j].
 cudaError_t launch_gather_layernorm(bool half_out, const float* src, int src_rows, const int32_t* idx,
                                     int B, int n, int D, const float* gamma, const float* beta, float eps,
-                                    float* x_out, void* u_out, cudaStream_t st);
+                                    float* x_out, void* u_out, cudaStream_t st, const int32_t* out_idx = nullptr,
+                                    int out_rows = 0);
 
 // K5: K/V write-back into one block's cache slice [2][B][S][D]; idx NULL = identity.
 cudaError_t launch_scatter_kv(bool bf16_t, const void* k, const void* v, int ld_kv, const int32_t* idx,
@@ -24,6 +25,14 @@ cudaError_t launch_scatter_rows(const float* rows, const int32_t* idx, int B, in
 // fp32 row gather out[b][j] = src[b][idx[b][j]].
 cudaError_t launch_gather_rows(const float* src, const int32_t* idx, int B, int n, int S, int D, float* out,
                                cudaStream_t st);
+
+// out[r] = table[idx[r]] for total_rows rows of D floats (table shared by all samples).
+cudaError_t launch_gather_table_rows(const float* table, const int32_t* idx, long total_rows, int D, float* out,
+                                     cudaStream_t st);
+
+// out[b][s] = mask_token + pos[s], float [B][S][D] (Eq. 2, masked positions of the decoder's input).
+cudaError_t launch_fill_mask_rows(const float* mask_token, const float* pos, int B, int S, int D, float* out,
+                                  cudaStream_t st);
 
 // a0 prologue: is_new[b][j] (may be NULL with n_active = 0) and the candidate mask cand[b][t].
 cudaError_t launch_step_flags(const int32_t* active_idx, int n_active, const int32_t* new_idx, int n_new,

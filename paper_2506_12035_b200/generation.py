@@ -113,6 +113,46 @@ class Generation:
             m.scatter_rows(self.rows[t], G, self.hidden, stream)
         return log
 
+    # ------------------------------------------------------------------ two-stage model (Eq. 1, Eq. 2)
+    def run_mar(self, tokens0: torch.Tensor, known_sets: Sequence, budget: int = 64, period: int = 3,
+                record: bool = False, forced_refresh: Optional[List[Optional[torch.Tensor]]] = None, stream=None,
+                n_steps: Optional[int] = None, mode: str = "marche"):
+        """Encoder over the known tokens and cache-aware decoder, Section 4.3 schedule: the decoder is
+        fully refreshed at t = 0 and every `period`-th step (always with mode "full"), otherwise it
+        runs the in-step selection with K = budget - #G - #N.  known_sets[t]: int32 [B][n_known(t)].
+        The decoder outputs land in self.hidden_out."""
+        m, B, S = self.m, self.m.B, self.m.S
+        if not hasattr(self, "known_sets_dev") or len(self.known_sets_dev) != len(known_sets):
+            self.known_sets_dev = [torch.as_tensor(k, dtype=torch.int32).to("cuda").contiguous() for k in known_sets]
+        self.hidden.copy_(tokens0, non_blocking=True)
+        m.init_cache(self.cache, stream)
+        log = []
+        for t in range(self.T if n_steps is None else min(n_steps, self.T)):
+            G = self.new_sets[t]
+            N = self.new_sets[t - 1] if t > 0 else None
+            Kn = self.known_sets_dev[t]
+            if mode == "full" or t % period == 0:
+                m.mar_step(True, self.hidden, Kn, self.cache, G, N, 0, None, self.hidden_out, None, None,
+                           self.workspace, stream)
+                n_active, k, active = S, 0, None
+            else:
+                n_gn = G.shape[1] + N.shape[1]
+                k = min(max(0, budget - n_gn), S - n_gn)
+                n_active = n_gn + k
+                active = self.active_flat[: B * n_active].view(B, n_active)
+                fr = None if forced_refresh is None else forced_refresh[t]
+                m.mar_step(False, self.hidden, Kn, self.cache, G, N, k, fr, self.hidden_out, self.refresh_flat[0],
+                           active, self.workspace, stream)
+            if record:
+                m.get_scores(self.workspace, self.scores, stream)
+                torch.cuda.synchronize()
+                log.append(dict(t=t, n_active=n_active, active=None if active is None else active.cpu().numpy().copy(),
+                                scores=self.scores.cpu().numpy().copy(),
+                                refresh=self.refresh_flat[0][: B * k].view(B, k).cpu().numpy().copy(),
+                                z=self.hidden_out.cpu().numpy().copy()))
+            m.scatter_rows(self.rows[t], G, self.hidden, stream)
+        return log
+
     # ------------------------------------------------------------------ host-driven loop
     def alloc_host_buffers(self, hidden0, rows_np, sets_np):
         """Pinned host buffers for run_host: the stack input, per step the sampled rows and

@@ -101,3 +101,90 @@ def test_full_size_sampled_parity(name):
     assert max_abs(Kc, cache2.K) <= ma and rel_l2(Kc, cache2.K) <= rl
     assert max_abs(Vc, cache2.V) <= ma and rel_l2(Vc, cache2.V) <= rl
     print("full-size parity: hidden max-abs %.3g, cache K max-abs %.3g" % (worst, max_abs(Kc, cache2.K)))
+
+
+def test_full_size_two_stage_sampled_parity():
+    """The two-stage step (encoder over the known tokens, cache-aware decoder) at the MAR-L shape and
+    batch 128: a full-decoder step and two in-step-selection steps with the fixed budget of 64,
+    the oracle on one guidance pair, teacher-forced for that pair."""
+    from paper_2506_12035_b200.binding import upload_mar_weights
+    cfg = synth.CONFIGS["mar_l"]
+    if torch.cuda.get_device_properties(0).total_memory < 40e9:
+        pytest.skip("needs a large GPU")
+    pair = [0, cfg.B // 2]
+    budget, n_steps = 64, 3
+    blocks = synth.make_weights(cfg)
+    mar = synth.make_mar_weights(cfg)
+    m = make_model(cfg, blocks)
+    m.set_mar_weights(upload_mar_weights(mar, cfg.dtype))
+    tokens_np = synth.make_hidden(cfg)
+    sets = synth.new_token_sets(cfg, synth.generation_orders(cfg))
+    known = synth.known_token_sets(cfg, sets)
+
+    # ---- oracle on the pair
+    t2 = tokens_np[pair].copy()
+    s2 = [g[pair] for g in sets]
+    k2 = [k[pair] for k in known]
+    cache2 = orc.KVCache(cfg.L, 2, cfg.S, cfg.D)
+    z2 = np.zeros_like(t2)
+    kw = dict(n_heads=cfg.H, n_enc=cfg.E, score_layer=cfg.score_layer, ln_eps=cfg.ln_eps)
+    recs = []
+    for t in range(n_steps):
+        if t > 0:
+            rows = synth.replacement_rows(cfg, t - 1, s2[t - 1].shape[1], batch=cfg.B)[pair]
+            for i in range(2):
+                t2[i, s2[t - 1][i]] = rows[i]
+        N = s2[t - 1] if t > 0 else None
+        kk = 0 if t == 0 else budget - s2[t].shape[1] - s2[t - 1].shape[1]
+        sc, R, A = orc.mar_step(blocks, mar, t2, k2[t], cache2, s2[t], N, kk, z2, full_decoder=(t == 0), **kw)
+        recs.append(dict(active=A, z=z2.copy(), scores=sc, refresh=R))
+    del blocks
+
+    # ---- device on the whole batch
+    B, S, D = cfg.B, cfg.S, cfg.D
+    tokens = dev(tokens_np)
+    z = torch.zeros(B, S, D, device="cuda")
+    cache = m.alloc_cache()
+    ws = m.alloc_workspace(S)
+    m.init_cache(cache)
+    scores = torch.empty(B, S, device="cuda")
+    ma, rl = TOL["bf16"]
+    worst = 0.0
+    for t in range(n_steps):
+        G, Kn = idx_dev(sets[t]), idx_dev(known[t])
+        rec = recs[t]
+        if t == 0:
+            m.mar_step(True, tokens, Kn, cache, G, None, 0, None, z, None, None, ws)
+        else:
+            N = idx_dev(sets[t - 1])
+            m.scatter_rows(dev(synth.replacement_rows(cfg, t - 1, sets[t - 1].shape[1])), N, tokens)
+            k = budget - sets[t].shape[1] - sets[t - 1].shape[1]
+            refresh = torch.empty(B, k, dtype=torch.int32, device="cuda")
+            active = torch.empty(B, budget, dtype=torch.int32, device="cuda")
+            # The device's own selection for the rows the oracle does not cover: a pre-pass with no
+            # refreshing tokens leaves the relevance scores in the workspace.  It rewrites only cache
+            # rows of G u N, which the real step rewrites again from inputs the pre-pass did not touch.
+            m.mar_step(False, tokens, Kn, cache, G, N, 0, None, torch.zeros_like(z), None,
+                       torch.empty(B, budget - k, dtype=torch.int32, device="cuda"), ws)
+            m.get_scores(ws, scores)
+            forced = torch.empty(B, k, dtype=torch.int32, device="cuda")
+            m.select_refresh(scores, G, N, k, forced, torch.empty(B * S, dtype=torch.uint8, device="cuda"))
+            forced[pair] = torch.as_tensor(rec["refresh"]).cuda()
+            m.mar_step(False, tokens, Kn, cache, G, N, k, forced, z, refresh, active, ws)
+            assert np.array_equal(active[pair].cpu().numpy(), rec["active"])
+        m.get_scores(ws, scores)
+        torch.cuda.synchronize()
+        assert m.device_status() == 0
+        got = z[pair].cpu().numpy()
+        for i in range(2):
+            a, w = got[i, rec["active"][i]], rec["z"][i, rec["active"][i]]
+            worst = max(worst, max_abs(a, w))
+            assert max_abs(a, w) <= ma and rel_l2(a, w) <= rl, \
+                "step %d sample %d: max-abs %.3g rel-L2 %.3g" % (t, pair[i], max_abs(a, w), rel_l2(a, w))
+        unit = cfg.H * sets[t].shape[1] / cfg.S
+        assert max_abs(scores[pair].cpu().numpy(), rec["scores"]) <= 5e-2 * unit
+    Kc = cache[cfg.E:, 0][:, pair].float().cpu().numpy()
+    Vc = cache[cfg.E:, 1][:, pair].float().cpu().numpy()
+    assert max_abs(Kc, cache2.K[cfg.E:]) <= ma and rel_l2(Kc, cache2.K[cfg.E:]) <= rl
+    assert max_abs(Vc, cache2.V[cfg.E:]) <= ma and rel_l2(Vc, cache2.V[cfg.E:]) <= rl
+    print("two-stage full-size parity: z max-abs %.3g" % worst)
