@@ -143,6 +143,8 @@ def algorithmic_work(cfg, sched):
     B, S, D, F, L, H = cfg.B, cfg.S, cfg.D, cfg.F, cfg.L, cfg.H
     w = {"gemm_flops": 0.0, "attention_bytes": 0.0, "attention_flops": 0.0, "gather_layernorm_bytes": 0.0,
          "scatter_kv_bytes": 0.0, "scatter_rows_bytes": 0.0, "topk_bytes": 0.0}
+    w["gemm_split"] = {"gemm_qkv": 3.0 * D * D, "gemm_out_proj": 1.0 * D * D, "gemm_fc1_gelu": 1.0 * D * F,
+                       "gemm_fc2": 1.0 * D * F}
     for g, nA, k in sched:
         M = B * nA
         w["gemm_flops"] += 2.0 * M * (4 * D * D + 2 * D * F) * L
@@ -173,6 +175,13 @@ def kernel_table(prof, work, peaks, attention_bound):
 
     add("gemm_tcgen05 (qkv, out, fc1, fc2)", "tensor", work["gemm_flops"], sum(prof[c][0] for c in GEMM_CLASSES),
         sum(prof[c][1] for c in GEMM_CLASSES), peaks["bf16_tflops_sustained"], "TFLOP/s")
+    # the same row split by projection (flops in proportion 3 D^2 : D^2 : D F : D F)
+    if rows and "gemm_split" in work:
+        tot = sum(work["gemm_split"].values())
+        rows[-1]["by_projection"] = {
+            c: {"us_per_launch": 1e3 * prof[c][0] / prof[c][1],
+                "frac": work["gemm_flops"] * work["gemm_split"][c] / tot / (prof[c][0] * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"]}
+            for c in GEMM_CLASSES if prof[c][1]}
     if attention_bound == "hbm":
         add("attention", "hbm", work["attention_bytes"], *prof["attention"], peaks["hbm_gbs"], "GB/s")
     else:
