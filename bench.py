@@ -352,6 +352,17 @@ def run_ours(args, cfg):
                             "peak_source": "%s (%s)" % (peak_kind, "sustained bf16 GEMM" if dom["bound"] == "tensor" else "device copy"),
                             "timing": "CUDA events in front of every launch, cache-aware steps of one generation of the timed workload"}
 
+        # ---- per-step latency: events between the steps of one more generation
+        if n_dec is None:
+            evs = [torch.cuda.Event(enable_timing=True) for _ in range(cfg.T + 1)]
+            evs[0].record()
+            gen.run(hidden0, after_step=lambda t: evs[t + 1].record())
+            torch.cuda.synchronize()
+            lat = [evs[t].elapsed_time(evs[t + 1]) for t in range(cfg.T)]
+            line["step_latency_ms"] = {"full_step_t0": lat[0], "cache_aware_median": float(np.median(lat[1:])),
+                                       "cache_aware_min": float(np.min(lat[1:])), "cache_aware_max": float(np.max(lat[1:])),
+                                       "note": "includes the overwrite of the generated rows after each step"}
+
         # ---- each kernel on its own at the median cache-aware shape (no dependency gaps)
         n_mid = int(np.median([s_[1] for s_ in sched[1:]]))
         line["kernels_isolated"] = {"n_active": n_mid, "rows": isolated_kernels(m, cfg, peaks, n_mid)}
@@ -412,7 +423,7 @@ def run_ours(args, cfg):
 
 def isolated_kernels(m, cfg, peaks, n_active):
     """Each hot-path kernel timed on its own at one mid-run shape (n_active rows per sample):
-    back-to-back launches through the single-kernel C calls, CUDA events around the batch, buffers
+    back-to-back launches through the single-kernel C calls (replayed from a CUDA graph), CUDA events around the batch, buffers
     rotated so that streamed operands come from HBM.  Unlike the per-class table of the generation,
     these figures contain no dependency gaps: they are the kernels' own roofline fractions."""
     import torch
@@ -439,12 +450,22 @@ def isolated_kernels(m, cfg, peaks, n_active):
     new = idx[:, :4].contiguous()
 
     def timed_us(fn, reps=24):
+        # the launches are recorded into a CUDA graph and replayed, so that the host's per-call cost
+        # (several microseconds through the Python binding) does not bound the small kernels
         for i in range(3):
             fn(i)
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                for i in range(reps):
+                    fn(i)
+        graph.replay()
+        torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        for i in range(reps):
-            fn(i)
+        graph.replay()
         e1.record()
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) / reps * 1e3
@@ -517,6 +538,30 @@ def run_microbench(args):
                     "latency_change": res["two_segment_us"] / res["scatter_then_attend_us"] - 1.0,
                     "paper_reports": "-19.2 % at (32, 256) on its hardware, -16.2 .. -27.3 % overall"})
         print(json.dumps(res), flush=True)
+
+    # ---- K4 at scale: the per-step call (B 128) is latency-bound and cannot show a bandwidth figure, so
+    # the same two kernels (candidate flags, radix select) are also run on many samples.
+    peaks, _ = load_peaks()
+    for Bk, Sk, k in ((128, 320, 32), (16384, 320, 32), (16384, 1088, 109)):
+        small = synth.CONFIGS["tiny"].replace(L=1, E=0, D=128, H=2, F=128, S=Sk, B=Bk, dtype="bf16")
+        m = Marche.from_config(small, upload_weights(synth.make_weights(small), "bf16"))
+        scores = torch.rand(Bk, Sk, device="cuda")
+        new = torch.stack([torch.randperm(Sk, device="cuda")[:4] for _ in range(min(Bk, 256))]).to(torch.int32)
+        new = new.repeat((Bk + new.shape[0] - 1) // new.shape[0], 1)[:Bk].contiguous()
+        out = torch.empty(Bk, k, dtype=torch.int32, device="cuda")
+        mask = torch.empty(Bk * Sk, dtype=torch.uint8, device="cuda")
+        for _ in range(3):
+            m.select_refresh(scores, new, None, k, out, mask)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(10):
+            m.select_refresh(scores, new, None, k, out, mask)
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) / 10 * 1e3
+        nbytes = Bk * Sk * 5 + Bk * k * 4 + Bk * Sk          # scores + mask read, indices written, mask written
+        print(json.dumps({"microbench": "top-k refresh selection (flags + radix select)", "batch": Bk, "seq_len": Sk, "k": k,
+                          "us": us, "GB/s": nbytes / us * 1e-3, "frac_of_hbm": nbytes / us * 1e-3 / peaks["hbm_gbs"]}), flush=True)
 
 
 def main():

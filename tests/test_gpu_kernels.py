@@ -270,7 +270,8 @@ def test_attention_uniform_and_peaked(dtype):
 
 
 # ------------------------------------------------------------------ K4 top-k (bit-exact)
-@pytest.mark.parametrize("S,k", [(5, 2), (68, 7), (320, 32), (320, 0), (320, 311), (1088, 109), (1088, 1)])
+@pytest.mark.parametrize("S,k", [(5, 2), (68, 7), (320, 32), (320, 0), (320, 311), (1088, 109), (1088, 1), (2048, 205),
+                                 (2048, 2043), (33, 28)])
 def test_select_refresh_bit_exact(S, k):
     B = 4
     cfg, blocks, m = model_for("f32", 128, 2, 128, S, B)
