@@ -304,6 +304,18 @@ int marche_select_refresh_static(marche_ctx* ctx, const float* scores,
  * from the generating tokens to each token, summed over heads and queries. */
 int marche_get_scores(marche_ctx* ctx, const void* workspace, float* scores_out, marche_stream stream);
 
+/* Relevance scores at more than one block (the top-K overlap statistics across decoder layers of
+ * Section 5.3 / Appendix G need them).  marche_set_score_layers registers up to 64 blocks that
+ * accumulate scores in addition to score_layer (which alone drives the selection); it changes the
+ * workspace size, so call it before marche_workspace_bytes.  n = 0 clears the list.  The extra
+ * blocks are honoured by marche_step and marche_full_step, and by the every-token phase of
+ * marche_step_in_step_selection / marche_mar_step (full decoder only); each costs the two-pass
+ * scoring variant of the attention kernel.  marche_get_layer_scores sums the per-head partials of
+ * one registered block (or of score_layer) left in `workspace` by the last step, in head order,
+ * into scores_out, device float [B][S].  MARCHE_EINVAL for a block that is not registered. */
+int marche_set_score_layers(marche_ctx* ctx, const int32_t* layers /* host */, int n);
+int marche_get_layer_scores(marche_ctx* ctx, void* workspace, int layer, float* scores_out, marche_stream stream);
+
 /* Algorithm 1 line 4, A = G u N u R, built on the device so that a generation
  * loop needs no host round trip: active_idx[b] = new_idx[b] | prev_idx[b] |
  * refresh_idx[b] (concatenation; the caller guarantees disjointness).  Any of

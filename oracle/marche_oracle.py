@@ -251,7 +251,8 @@ def _block(X, blk, K_l, V_l, idx, n_heads, eps, scoring_rows):
 def marche_step(blocks: Sequence[Block], hidden: np.ndarray, cache: KVCache,
                 active_idx: np.ndarray, new_idx: np.ndarray, exclude_idx: Optional[np.ndarray],
                 refresh_ratio: float, hidden_out: np.ndarray, *, n_heads: int, score_layer: int,
-                ln_eps: float = 1e-6, real=np.float64, require_filled: bool = True):
+                ln_eps: float = 1e-6, real=np.float64, require_filled: bool = True,
+                layer_scores: Optional[Dict[int, np.ndarray]] = None):
     """One cache-aware decoding step (Algorithm 1), every sample independently.
 
     hidden fp32 [B][S][D]; active_idx int32 [B][nA]; new_idx int32 [B][nG]
@@ -259,6 +260,9 @@ def marche_step(blocks: Sequence[Block], hidden: np.ndarray, cache: KVCache,
     exclude_idx int32 [B][nX] or None.  Rows `active_idx` of `hidden_out`
     ([B][S][D], modified in place) receive the stack output; every other row of
     `hidden_out` and of the cache keeps its bytes.
+    `layer_scores`, when given, is a dict whose keys are block indices; each value is replaced by
+    that block's relevance scores fp32 [B][S] (same definition as at score_layer; for the top-K
+    overlap statistics across layers of Section 5.3).
     Returns (scores fp32 [B][S], refresh_idx int32 [B][k])."""
     if require_filled and not cache.filled:
         raise RuntimeError("cache-aware step before any full step")
@@ -266,6 +270,7 @@ def marche_step(blocks: Sequence[Block], hidden: np.ndarray, cache: KVCache,
     L = len(blocks)
     blocks = [{k: np.asarray(v, dtype=real) for k, v in blk.items()} for blk in blocks]
     scores = np.zeros((B, S), dtype=real)
+    extra = {l: np.zeros((B, S), dtype=real) for l in (layer_scores or {})}
     for b in range(B):
         idx = np.asarray(active_idx[b], dtype=np.int64)
         if len(set(idx.tolist())) != len(idx) or idx.min() < 0 or idx.max() >= S:
@@ -276,12 +281,17 @@ def marche_step(blocks: Sequence[Block], hidden: np.ndarray, cache: KVCache,
         scoring_rows = np.array([int(t) in new for t in idx], dtype=bool)
         X = hidden[b, idx].astype(real)
         for l in range(L):
+            wanted = l == score_layer or (layer_scores is not None and l in layer_scores)
             X, sc = _block(X, blocks[l], cache.K[l, b], cache.V[l, b], idx, n_heads, ln_eps,
-                           scoring_rows if l == score_layer else None)
-            if sc is not None:
+                           scoring_rows if wanted else None)
+            if sc is not None and l == score_layer:
                 scores[b] = sc
+            if sc is not None and layer_scores is not None and l in layer_scores:
+                extra[l][b] = sc
         hidden_out[b, idx] = X.astype(hidden_out.dtype)
     scores32 = scores.astype(np.float32)
+    for l in extra:
+        layer_scores[l] = extra[l].astype(np.float32)
     n_new = new_idx.shape[1]
     n_excl = 0 if exclude_idx is None else exclude_idx.shape[1]
     k = refresh_count(refresh_ratio, S, S - n_new - n_excl)
@@ -289,14 +299,14 @@ def marche_step(blocks: Sequence[Block], hidden: np.ndarray, cache: KVCache,
 
 
 def full_step(blocks, hidden, cache: KVCache, new_idx, exclude_idx, refresh_ratio, hidden_out, *,
-              n_heads, score_layer, ln_eps=1e-6, real=np.float64):
+              n_heads, score_layer, ln_eps=1e-6, real=np.float64, layer_scores=None):
     """Every token active: fills the cache (initial full refresh, Section 4.3) and
     is the full-recompute baseline (every token recomputed at every step)."""
     B, S, _ = hidden.shape
     all_idx = np.tile(np.arange(S, dtype=np.int32), (B, 1))
     out = marche_step(blocks, hidden, cache, all_idx, new_idx, exclude_idx, refresh_ratio, hidden_out,
                       n_heads=n_heads, score_layer=score_layer, ln_eps=ln_eps, real=real,
-                      require_filled=False)
+                      require_filled=False, layer_scores=layer_scores)
     cache.filled = True
     return out
 

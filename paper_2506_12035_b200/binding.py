@@ -64,6 +64,8 @@ _SIGNATURES = {
     "marche_select_refresh_policy": (C.c_int, [_vp, _vp, _vp, _i, _vp, _i, _i, _i, C.c_uint32, _vp, _vp, _vp]),
     "marche_select_refresh_static": (C.c_int, [_vp, _vp, _vp, _i, _vp, _i, _i, _vp, _vp]),
     "marche_get_scores": (C.c_int, [_vp, _vp, _vp, _vp]),
+    "marche_set_score_layers": (C.c_int, [_vp, C.POINTER(C.c_int32), _i]),
+    "marche_get_layer_scores": (C.c_int, [_vp, _vp, _i, _vp, _vp]),
     "marche_build_active": (C.c_int, [_vp, _vp, _i, _vp, _i, _vp, _i, _vp, _vp]),
     "marche_scatter_rows": (C.c_int, [_vp, _vp, _vp, _i, _vp, _vp]),
     "marche_validate_indices": (C.c_int, [_vp, _vp, _i, _vp, _i, _vp, _i, _vp]),
@@ -280,6 +282,13 @@ class Marche:
 
     def get_scores(self, workspace, scores_out, stream=None):
         self._check(self.lib.marche_get_scores(self.h, _ptr(workspace), _ptr(scores_out), _stream(stream)))
+
+    def set_score_layers(self, layers: Sequence[int]):
+        arr = (C.c_int32 * max(len(layers), 1))(*layers)
+        self._check(self.lib.marche_set_score_layers(self.h, arr, len(layers)))
+
+    def get_layer_scores(self, workspace, layer: int, scores_out, stream=None):
+        self._check(self.lib.marche_get_layer_scores(self.h, _ptr(workspace), layer, _ptr(scores_out), _stream(stream)))
 
     def build_active(self, new_idx, prev_idx, refresh_idx, n_refresh, active_idx, stream=None):
         self._check(self.lib.marche_build_active(

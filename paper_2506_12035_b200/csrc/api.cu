@@ -34,6 +34,7 @@ struct marche_ctx {
   size_t eb = 4;
   float eps = 1e-6f;
   int score_layer = 0;
+  std::vector<int> extra_score_layers;                // blocks that also accumulate scores (analysis only)
   bool force_simt = false;
   bool stream_k = true;                               // MARCHE_STREAM_K=0: whole tiles only in the residual GEMMs
   bool fuse_writeback = false;                        // MARCHE_FUSE_WB=1: write-back fused into the attention prologue
@@ -67,7 +68,7 @@ WsLayout ws_layout(const marche_ctx* c, int nA) {
   WsLayout w;
   size_t off = 0;
   w.scores = off;  off += align256(B * S * sizeof(float));
-  w.partial = off; off += align256(B * H * S * sizeof(float));
+  w.partial = off; off += align256((1 + c->extra_score_layers.size()) * B * H * S * sizeof(float));
   w.cand = off;    off += align256(B * S);
   w.is_new = off;  off += align256(M);
   w.turn_bytes = gemm_tcgen05_2cta_turn_bytes((int)M, (int)D);   // stream-K turn flags of the residual GEMMs
@@ -112,6 +113,15 @@ void mark(marche_ctx* ctx, int cls, cudaStream_t st) {
 int refresh_count(float ratio, int S, int n_cand) {
   const int want = (int)std::floor((double)ratio * (double)S + 0.5);
   return want < n_cand ? (want < 0 ? 0 : want) : n_cand;
+}
+
+// Slot of block l in the per-head score partials: 0 = the scoring block that drives the selection,
+// 1.. = the extra analysis blocks, -1 = this block accumulates no scores.
+int score_slot(const marche_ctx* ctx, int l) {
+  if (l == ctx->score_layer) return 0;
+  for (size_t i = 0; i < ctx->extra_score_layers.size(); ++i)
+    if (ctx->extra_score_layers[i] == l) return (int)i + 1;
+  return -1;
 }
 
 int do_linear(marche_ctx* ctx, int cls, const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
@@ -199,6 +209,9 @@ int run_blocks(marche_ctx* ctx, int l_begin, int l_end, const float* gather_src,
   for (int l = l_begin; l < l_end; ++l) {
     const marche_block_weights& bw = ctx->blocks[l];
     char* cache_l = (char*)kv_cache + (size_t)l * layer_bytes;
+    const int slot = is_new ? score_slot(ctx, l) : -1;
+    const uint8_t* flags_l = slot >= 0 ? is_new : nullptr;
+    float* partial_l = bf.partial + (size_t)(slot > 0 ? slot : 0) * B * c.n_heads * c.seq_len;
     mark(ctx, MARCHE_KC_GATHER_LN, st);
     if (l == l_begin && gather_src)
       MARCHE_TRY(launch_gather_layernorm(ctx->bf16, gather_src, src_rows, idx, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
@@ -212,21 +225,21 @@ int run_blocks(marche_ctx* ctx, int l_begin, int l_end, const float* gather_src,
       // two-segment attention: fresh K/V read in place, cache write-back by the same kernel
       mark(ctx, MARCHE_KC_ATTENTION, st);
       MARCHE_TRY(launch_attention_twoseg(bf.qkv, 3 * D, D, 2 * D, B, nA, S, c.n_heads, c.head_dim, kv_idx, cache_l,
-                                         l == ctx->score_layer ? is_new : nullptr, bf.partial, bf.o, ctx->status_dev, st),
+                                         flags_l, partial_l, bf.o, ctx->status_dev, st),
                  "attention_twoseg");
     } else if (ctx->fuse_writeback && ctx->bf16 && !ctx->force_simt && ctx->attn_tc != 1 &&
                !(c.head_dim == 64 && ctx->attn_tc < 0 &&
-                 nA > ((l == ctx->score_layer && is_new) ? 64 : ctx->attn_tc_min_rows))) {
+                 nA > (flags_l ? 64 : ctx->attn_tc_min_rows))) {
       // mma.sync attention with the cache write-back fused into its prologue (no scatter_kv launch)
       mark(ctx, MARCHE_KC_ATTENTION, st);
       MARCHE_TRY(launch_attention_mma(bf.qkv, 3 * D, B, nA, S, c.n_heads, c.head_dim, cache_l,
-                                      l == ctx->score_layer ? is_new : nullptr, bf.partial, bf.o, ctx->status_dev, st,
+                                      flags_l, partial_l, bf.o, ctx->status_dev, st,
                                       true, kv_idx, D, 2 * D), "attention_mma_wb");
     } else {
       mark(ctx, MARCHE_KC_SCATTER_KV, st);
       MARCHE_TRY(launch_scatter_kv(ctx->bf16, bf.qkv + (size_t)D * eb, bf.qkv + (size_t)2 * D * eb, 3 * D, kv_idx, B, nA,
                                    S, D, cache_l, st), "scatter_kv");
-      rc = do_attention(ctx, bf.qkv, 3 * D, nA, cache_l, l == ctx->score_layer ? is_new : nullptr, bf.partial, bf.o, st,
+      rc = do_attention(ctx, bf.qkv, 3 * D, nA, cache_l, flags_l, partial_l, bf.o, st,
                         S);
       if (rc) return rc;
     }
@@ -556,6 +569,33 @@ int marche_select_refresh_policy(marche_ctx* ctx, const float* scores, const int
   mark(ctx, MARCHE_KC_TOPK, st);
   MARCHE_TRY(launch_topk(nullptr, 0, const_cast<float*>(scores), (const uint8_t*)mask_scratch, B, S, k, refresh_idx,
                          st, policy, seed), "topk");
+  return MARCHE_OK;
+}
+
+int marche_set_score_layers(marche_ctx* ctx, const int32_t* layers, int n) {
+  if (!ctx || n < 0 || n > 64 || (n > 0 && !layers)) return MARCHE_EINVAL;
+  std::vector<int> v;
+  for (int i = 0; i < n; ++i) {
+    if (layers[i] < 0 || layers[i] >= ctx->cfg.n_blocks) return MARCHE_EINVAL;
+    bool dup = layers[i] == ctx->score_layer;
+    for (int x : v) dup = dup || x == layers[i];
+    if (!dup) v.push_back(layers[i]);
+  }
+  ctx->extra_score_layers = v;
+  return MARCHE_OK;
+}
+
+int marche_get_layer_scores(marche_ctx* ctx, void* workspace, int layer, float* scores_out, marche_stream stream) {
+  if (!ctx || !workspace || !scores_out) return MARCHE_EINVAL;
+  const int slot = score_slot(ctx, layer);
+  if (slot < 0) return MARCHE_EINVAL;
+  const marche_config& c = ctx->cfg;
+  const WsLayout w = ws_layout(ctx, 1);
+  const float* partial = (const float*)((const char*)workspace + w.partial) + (size_t)slot * c.batch * c.n_heads * c.seq_len;
+  mark(ctx, MARCHE_KC_TOPK, (cudaStream_t)stream);
+  // k = 0: the kernel only adds the per-head partials in head order and writes the sums
+  MARCHE_TRY(launch_topk(partial, c.n_heads, scores_out, nullptr, c.batch, c.seq_len, 0, nullptr, (cudaStream_t)stream),
+             "score_sum");
   return MARCHE_OK;
 }
 

@@ -266,3 +266,68 @@ def test_argument_errors():
     with pytest.raises(MarcheError) as e:                                       # width not a multiple of 128
         Marche(L=1, E=0, D=192, H=3, F=128, S=8, B=1, dtype="f32", weights=upload_weights(blocks[:1], "f32"))
     assert e.value.code == -2
+
+
+@pytest.mark.parametrize("case", ["tiny_f32", "marb_slice"])
+def test_scores_at_several_blocks(case):
+    """Extra scoring blocks (for the top-K overlap statistics across layers): each block's scores
+    match the oracle's, the step's outputs and its selection do not change, and the overlap of the
+    per-block top-K sets can be computed from them."""
+    cfg = CASES[case]
+    blocks = synth.make_weights(cfg)
+    hidden0 = synth.make_hidden(cfg)
+    sets = synth.new_token_sets(cfg, synth.generation_orders(cfg))
+    G, X = sets[0], sets[1]
+    layers = list(range(cfg.L))
+    want = {l: None for l in layers}
+    cache_o = orc.KVCache(cfg.L, cfg.B, cfg.S, cfg.D)
+    out_o = np.zeros_like(hidden0)
+    s_o, r_o = orc.full_step(blocks, hidden0, cache_o, G, X, cfg.ratio, out_o, n_heads=cfg.H, score_layer=cfg.score_layer,
+                             ln_eps=cfg.ln_eps, layer_scores=want)
+
+    m_plain = make_model(cfg, blocks)
+    m = make_model(cfg, blocks)
+    ws_plain = m_plain.alloc_workspace(cfg.S)
+    m.set_score_layers(layers)
+    ws = m.alloc_workspace(cfg.S)
+    assert ws.numel() > ws_plain.numel()
+    outs = []
+    for mm, w in ((m_plain, ws_plain), (m, ws)):
+        cache = mm.alloc_cache()
+        mm.init_cache(cache)
+        out = torch.zeros(cfg.B, cfg.S, cfg.D, device="cuda")
+        refresh = torch.zeros(cfg.B * cfg.S, dtype=torch.int32, device="cuda")
+        k = mm.full_step(dev(hidden0), cache, idx_dev(G), idx_dev(X), cfg.ratio, out, refresh, w)
+        outs.append((out, refresh[: cfg.B * k].clone(), cache))
+    if cfg.dtype == "f32":      # one attention kernel: registering blocks changes nothing at all
+        assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2], outs[1][2])
+    else:                       # the scoring flavour of the tensor-core kernel is two-pass: same values within rounding
+        assert_close(host(outs[1][0]), host(outs[0][0]), cfg.dtype, "outputs with extra scoring blocks")
+    assert_close(host(outs[1][0]), out_o, cfg.dtype, "outputs vs oracle")
+    unit = cfg.H * G.shape[1] / cfg.S
+    lim = (5e-2 if cfg.dtype == "bf16" else 1e-4) * unit
+    sc = torch.empty(cfg.B, cfg.S, device="cuda")
+    per_layer = {}
+    for l in layers:
+        m.get_layer_scores(ws, l, sc)
+        per_layer[l] = sc.cpu().numpy().copy()
+        assert max_abs(per_layer[l], want[l]) <= lim, l
+        assert np.allclose(per_layer[l].sum(-1), cfg.H * G.shape[1], rtol=2e-3)
+    m.get_scores(ws, sc)
+    assert np.array_equal(sc.cpu().numpy(), per_layer[cfg.score_layer])
+    # top-K overlap between two blocks from the device's scores, via the device's selection
+    k = 7
+    mask = torch.empty(cfg.B * cfg.S, dtype=torch.uint8, device="cuda")
+    tops = []
+    for l in (layers[0], layers[-1]):
+        out = torch.empty(cfg.B, k, dtype=torch.int32, device="cuda")
+        m.select_refresh(dev(per_layer[l]), idx_dev(G), None, k, out, mask)
+        assert np.array_equal(out.cpu().numpy(), orc.select_refresh(per_layer[l], G, None, k))
+        tops.append(out.cpu().numpy())
+    overlap = np.mean([len(set(a) & set(b)) / k for a, b in zip(*tops)])
+    assert 0.0 <= overlap <= 1.0
+    # a block that was not registered is refused; clearing the list restores the plain workspace size
+    with pytest.raises(MarcheError):
+        m_plain.get_layer_scores(ws_plain, (cfg.score_layer + 1) % cfg.L, sc)
+    m.set_score_layers([])
+    assert m.workspace_bytes(cfg.S) == m_plain.workspace_bytes(cfg.S)

@@ -493,3 +493,40 @@ def test_active_set_union():
     assert orc.active_set(G, N, R).tolist() == [[3, 4, 7, 0, 9]]
     with pytest.raises(ValueError):
         orc.active_set(G, N, np.array([[4, 9]], np.int32))
+
+
+def test_layer_scores_match_the_scoring_block_and_closed_forms():
+    """Scores requested at several blocks: at block l they are what a run with score_layer = l
+    returns; each obeys the checksum H * #G; a block with zero query weights gives H * #G / S."""
+    cfg = small_cfg()
+    blocks, hidden = setup(cfg)
+    D = cfg.D
+    blocks[2]["w_qkv"][:D] = 0
+    blocks[2]["b_qkv"][:D] = 0
+    G = np.array([[5, 9, 11], [4, 6, 19]], dtype=np.int32)
+    per_layer = []
+    for l in range(cfg.L):
+        cache = orc.KVCache(cfg.L, cfg.B, cfg.S, D)
+        s, _ = orc.full_step(blocks, hidden, cache, G, None, 0.0, np.zeros_like(hidden), n_heads=cfg.H, score_layer=l)
+        per_layer.append(s)
+    want = {0: None, 1: None, 2: None}
+    cache = orc.KVCache(cfg.L, cfg.B, cfg.S, D)
+    out_a = np.zeros_like(hidden)
+    main, ref_a = orc.full_step(blocks, hidden, cache, G, None, 0.2, out_a, n_heads=cfg.H, score_layer=1, layer_scores=want)
+    for l in range(cfg.L):
+        assert np.array_equal(want[l], per_layer[l])
+        assert np.allclose(want[l].sum(-1), cfg.H * G.shape[1], rtol=1e-6)
+    assert np.array_equal(main, per_layer[1])
+    assert np.allclose(want[2], cfg.H * G.shape[1] / cfg.S, rtol=1e-6)
+    assert not np.allclose(want[0], want[1])
+    # asking for extra blocks changes neither the outputs nor the selection
+    cache_b = orc.KVCache(cfg.L, cfg.B, cfg.S, D)
+    out_b = np.zeros_like(hidden)
+    main_b, ref_b = orc.full_step(blocks, hidden, cache_b, G, None, 0.2, out_b, n_heads=cfg.H, score_layer=1)
+    assert np.array_equal(out_a, out_b) and np.array_equal(ref_a, ref_b) and np.array_equal(cache.K, cache_b.K)
+    # cache-aware step: same property on the active rows' queries
+    A = np.concatenate([G, np.array([[0, 1], [2, 3]], np.int32)], axis=1)
+    w2 = {0: None, 2: None}
+    s2, _ = orc.marche_step(blocks, hidden, cache, A, G, None, 0.0, out_a, n_heads=cfg.H, score_layer=1, layer_scores=w2)
+    assert np.allclose(w2[0].sum(-1), cfg.H * G.shape[1], rtol=1e-6)
+    assert np.allclose(w2[2], cfg.H * G.shape[1] / cfg.S, rtol=1e-6)
