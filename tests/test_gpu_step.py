@@ -331,3 +331,90 @@ def test_scores_at_several_blocks(case):
         m_plain.get_layer_scores(ws_plain, (cfg.score_layer + 1) % cfg.L, sc)
     m.set_score_layers([])
     assert m.workspace_bytes(cfg.S) == m_plain.workspace_bytes(cfg.S)
+
+
+def _one_step_pair(cfg, blocks, hidden0, G0, A, G, X, ratio):
+    """Full step then one cache-aware step on both sides; returns (oracle, device) results."""
+    kw = dict(n_heads=cfg.H, score_layer=cfg.score_layer, ln_eps=cfg.ln_eps)
+    cache_o = orc.KVCache(cfg.L, cfg.B, cfg.S, cfg.D)
+    out_o = np.zeros_like(hidden0)
+    orc.full_step(blocks, hidden0, cache_o, G0, None, ratio, out_o, **kw)
+    full_o = out_o.copy()
+    s_o, r_o = orc.marche_step(blocks, hidden0, cache_o, A, G, X, ratio, out_o, **kw)
+    m = make_model(cfg, blocks)
+    cache = m.alloc_cache()
+    ws = m.alloc_workspace(cfg.S)
+    m.init_cache(cache)
+    out = torch.zeros(cfg.B, cfg.S, cfg.D, device="cuda")
+    refresh = torch.full((cfg.B * cfg.S,), -1, dtype=torch.int32, device="cuda")
+    h = dev(hidden0)
+    m.full_step(h, cache, idx_dev(G0), None, ratio, out, refresh, ws)
+    full_d = out.cpu().numpy().copy()
+    k = m.step(h, cache, idx_dev(A), None if G.shape[1] == 0 else idx_dev(G), None if X is None else idx_dev(X), ratio,
+               out, refresh, ws)
+    sc = torch.empty(cfg.B, cfg.S, device="cuda")
+    m.get_scores(ws, sc)
+    torch.cuda.synchronize()
+    assert m.device_status() == 0
+    return (full_o, out_o, s_o, r_o, cache_o), (full_d, out.cpu().numpy(), sc.cpu().numpy(),
+                                                 refresh[: cfg.B * k].view(cfg.B, k).cpu().numpy(), cache)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_degenerate_active_sets(dtype):
+    """One active token; no generating token at all (all scores zero, so the selection falls back
+    to the lowest-index candidates); an active set that is every token but one."""
+    cfg = synth.CONFIGS["tiny"].replace(dtype=dtype)
+    blocks = synth.make_weights(cfg)
+    hidden0 = synth.make_hidden(cfg)
+    B, S = cfg.B, cfg.S
+    G0 = np.array([[5, 9], [4, 6]], dtype=np.int32)
+    empty = np.zeros((B, 0), dtype=np.int32)
+    cases = [
+        (np.array([[17], [33]], np.int32), np.array([[17], [33]], np.int32), None, 0.1),          # nA = nG = 1
+        (np.array([[17, 3], [33, 8]], np.int32), empty, np.array([[0], [1]], np.int32), 0.1),     # nG = 0
+        (np.stack([np.delete(np.arange(S, dtype=np.int32), 11), np.delete(np.arange(S, dtype=np.int32), 60)]),
+         np.array([[1, 2, 3], [4, 5, 6]], np.int32), None, 0.0),                                   # nA = S - 1, k = 0
+    ]
+    for A, G, X, ratio in cases:
+        (fo, oo, so, ro, co), (fd, od, sd, rd, cd) = _one_step_pair(cfg, blocks, hidden0, G0, A, G, X, ratio)
+        for b in range(B):
+            assert_close(od[b, A[b]], oo[b, A[b]], dtype, "active rows")
+            rest = np.setdiff1d(np.arange(S), A[b])
+            assert np.array_equal(od[b, rest], fd[b, rest])                # rows outside A keep the full step's bytes
+        unit = cfg.H * max(G.shape[1], 1) / S
+        assert max_abs(sd, so) <= (5e-2 if dtype == "bf16" else 1e-4) * unit
+        assert rd.shape == ro.shape
+        if G.shape[1] == 0:
+            assert (sd == 0).all() and np.array_equal(rd, ro)              # ties -> lowest indices, bit-exact
+        K, V = cache_to_oracle_layout(cd)
+        assert_close(K, co.K, dtype, "cache K")
+        assert_close(V, co.V, dtype, "cache V")
+
+
+@pytest.mark.parametrize("shape", ["S2048", "D2048"])
+def test_maximum_sizes(shape):
+    """The largest sequence length and the largest width the library accepts (one block, bf16)."""
+    base = synth.CONFIGS["tiny"].replace(dtype="bf16", L=1, E=0, B=2, T=4)
+    cfg = base.replace(S=2048, n_buffer=64, D=128, H=2, F=256) if shape == "S2048" else \
+        base.replace(S=72, n_buffer=8, D=2048, H=32, F=2048)
+    blocks = synth.make_weights(cfg)
+    hidden0 = synth.make_hidden(cfg)
+    rng = np.random.default_rng(3)
+    perm = np.stack([rng.permutation(cfg.S) for _ in range(cfg.B)]).astype(np.int32)
+    G0, G, N = perm[:, :5], perm[:, 5:9], perm[:, 9:40]
+    A = np.concatenate([G, N], axis=1)
+    (fo, oo, so, ro, co), (fd, od, sd, rd, cd) = _one_step_pair(cfg, blocks, hidden0, G0, A, G, None, 0.05)
+    assert_close(fd, fo, "bf16", "full step")
+    for b in range(cfg.B):
+        assert_close(od[b, A[b]], oo[b, A[b]], "bf16", "active rows")
+    assert max_abs(sd, so) <= 5e-2 * cfg.H * G.shape[1] / cfg.S
+    assert rd.shape == ro.shape == (cfg.B, int(np.floor(0.05 * cfg.S + 0.5)))
+    K, V = cache_to_oracle_layout(cd)
+    assert_close(K, co.K, "bf16", "cache K")
+    assert_close(V, co.V, "bf16", "cache V")
+    m = make_model(cfg, blocks)
+    mask = torch.empty(cfg.B * cfg.S, dtype=torch.uint8, device="cuda")
+    out = torch.empty(cfg.B, rd.shape[1], dtype=torch.int32, device="cuda")
+    m.select_refresh(dev(so), idx_dev(G), None, rd.shape[1], out, mask)
+    assert np.array_equal(out.cpu().numpy(), ro)
