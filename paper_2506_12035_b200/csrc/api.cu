@@ -37,6 +37,7 @@ struct marche_ctx {
   std::vector<int> extra_score_layers;                // blocks that also accumulate scores (analysis only)
   bool force_simt = false;
   bool stream_k = true;                               // MARCHE_STREAM_K=0: whole tiles only in the residual GEMMs
+  bool fuse_qkv_scatter = true;                       // MARCHE_FUSE_QKV_SCATTER=0: separate scatter_kv launch
   bool fuse_writeback = false;                        // MARCHE_FUSE_WB=1: write-back fused into the attention prologue
                                                       // (measured slower: +11.7 us attention vs -10.5 us scatter_kv launch)
   int attn_tc = -1;                                   // -1 auto, 0 never, 1 always (MARCHE_ATTN_TC)
@@ -124,15 +125,24 @@ int score_slot(const marche_ctx* ctx, int l) {
   return -1;
 }
 
+// True when the QKV projection of M rows can write K and V into the cache itself (CTA-pair GEMM,
+// whole 256-column tiles per q / K / V range, 32-bit cache offsets): no scatter_kv launch then.
+bool qkv_scatter_fused(const marche_ctx* ctx, int M, int S) {
+  const marche_config& c = ctx->cfg;
+  return ctx->fuse_qkv_scatter && ctx->bf16 && !ctx->force_simt && ctx->attn_mode == 0 && !ctx->fuse_writeback &&
+         (ctx->gemm_mode == 2 || (ctx->gemm_mode == 0 && M > 128)) && c.width % 256 == 0 &&
+         (long)2 * c.batch * S * c.width < (1L << 31);
+}
+
 int do_linear(marche_ctx* ctx, int cls, const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
-              int epi, void* out, cudaStream_t st, int* turn = nullptr) {
+              int epi, void* out, cudaStream_t st, int* turn = nullptr, const KvScatter* kv = nullptr) {
   if (M > 0) mark(ctx, cls, st);
   const bool tc = ctx->bf16 && !ctx->force_simt && N % 128 == 0 && K % 64 == 0 && lda % 8 == 0 &&
                   (((uintptr_t)a | (uintptr_t)w | (uintptr_t)out) & 15) == 0;
   const bool pair = tc && (ctx->gemm_mode == 2 || (ctx->gemm_mode == 0 && M > 128));
   if (pair)
     MARCHE_TRY(launch_gemm_tcgen05_2cta(a, lda, M, w, bias, N, K, epi, out, ctx->status_dev, st,
-                                        ctx->stream_k ? turn : nullptr), "gemm_tcgen05_2cta");
+                                        ctx->stream_k ? turn : nullptr, kv), "gemm_tcgen05_2cta");
   else if (tc)
     MARCHE_TRY(launch_gemm_tcgen05(a, lda, M, w, bias, N, K, epi, out, ctx->status_dev, st), "gemm_tcgen05");
   else
@@ -219,9 +229,16 @@ int run_blocks(marche_ctx* ctx, int l_begin, int l_end, const float* gather_src,
     else
       MARCHE_TRY(launch_gather_layernorm(ctx->bf16, x, nA, nullptr, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
                                          nullptr, bf.u, st), "layernorm1");
-    int rc = do_linear(ctx, MARCHE_KC_GEMM_QKV, bf.u, D, M, bw.w_qkv, bw.b_qkv, 3 * D, D, MARCHE_EPI_BIAS, bf.qkv, st);
+    const bool fused_kv = qkv_scatter_fused(ctx, M, S);
+    const KvScatter kvs = {kv_idx, cache_l, nA, S, B, D};
+    int rc = do_linear(ctx, MARCHE_KC_GEMM_QKV, bf.u, D, M, bw.w_qkv, bw.b_qkv, 3 * D, D, fused_kv ? 4 : MARCHE_EPI_BIAS,
+                       bf.qkv, st, nullptr, fused_kv ? &kvs : nullptr);
     if (rc) return rc;
-    if (ctx->attn_mode == 1 && ctx->bf16 && !ctx->force_simt) {
+    if (fused_kv) {
+      // the projection's epilogue has written K and V into the cache (Algorithm 1 line 11)
+      rc = do_attention(ctx, bf.qkv, 3 * D, nA, cache_l, flags_l, partial_l, bf.o, st, S);
+      if (rc) return rc;
+    } else if (ctx->attn_mode == 1 && ctx->bf16 && !ctx->force_simt) {
       // two-segment attention: fresh K/V read in place, cache write-back by the same kernel
       mark(ctx, MARCHE_KC_ATTENTION, st);
       MARCHE_TRY(launch_attention_twoseg(bf.qkv, 3 * D, D, 2 * D, B, nA, S, c.n_heads, c.head_dim, kv_idx, cache_l,
@@ -428,6 +445,8 @@ int marche_create(const marche_config* cfg, const marche_block_weights* blocks, 
   ctx->force_simt = fs && fs[0] == '1';
   const char* sk = getenv("MARCHE_STREAM_K");
   ctx->stream_k = !(sk && sk[0] == '0');
+  const char* fq = getenv("MARCHE_FUSE_QKV_SCATTER");
+  ctx->fuse_qkv_scatter = !(fq && fq[0] == '0');
   const char* fw = getenv("MARCHE_FUSE_WB");
   ctx->fuse_writeback = fw && fw[0] == '1';
   const char* tcv = getenv("MARCHE_ATTN_TC");

@@ -6,8 +6,11 @@
 //   EPI 0: out bf16 = acc + bias
 //   EPI 1: out fp32 += acc + bias   -- TMA reduce-add in L2, no read in the SM, one add per element
 //   EPI 2: out fp16 = GELU_erf(acc + bias)   (feeds the next projection as its A operand)
+//   EPI 4: as EPI 0 for the q columns; the K and V columns go straight into scattered rows of the
+//          K/V cache (epilogue_box_scatter), so no separate write-back launch is needed
 #pragma once
 
+#include "kernels.h"
 #include "sm100_ptx.cuh"
 
 namespace marche {
@@ -67,6 +70,48 @@ MARCHE_DEVINL void epilogue_box(uint32_t t_addr, const float* __restrict__ bias_
     else ptx::tma_store_2d(out_map, col, row0, stage);
     ptx::bulk_commit();
   }
+}
+
+// 64 bf16 columns of 32 accumulator rows, written straight into scattered cache rows.  The values
+// are staged through the warp's swizzled 4 KB box exactly as for the TMA store; then every quarter
+// warp copies one whole 128-byte row piece per instruction (lane l: chunk l % 8 of row l / 8 + 4 i), so
+// each global store instruction of the warp writes four full 128-byte lines.  dst_elem = element
+// offset of this lane's row in the cache plus the column of this box, or -1 for a row beyond M.
+MARCHE_DEVINL void epilogue_box_scatter(uint32_t t_addr, const float* __restrict__ bias_col, bf16* cache, int dst_elem,
+                                        uint32_t stage, int lane) {
+  if (lane == 0) ptx::bulk_wait_read_all();            // an earlier TMA store of this warp may still read the box
+  __syncwarp();
+  const uint32_t row_base = stage + (uint32_t)lane * 128u;
+  const float4* b4 = reinterpret_cast<const float4*>(bias_col);
+#pragma unroll
+  for (int hh = 0; hh < 2; ++hh) {
+    uint32_t r[32];
+    ptx::tmem_ld_32x32(t_addr + (uint32_t)(hh * 32), r);
+    ptx::tmem_ld_wait();
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float4 b0 = __ldg(b4 + hh * 8 + 2 * j), b1 = __ldg(b4 + hh * 8 + 2 * j + 1);
+      const uint32_t p0 = pack_bf16x2(__uint_as_float(r[8 * j + 0]) + b0.x, __uint_as_float(r[8 * j + 1]) + b0.y);
+      const uint32_t p1 = pack_bf16x2(__uint_as_float(r[8 * j + 2]) + b0.z, __uint_as_float(r[8 * j + 3]) + b0.w);
+      const uint32_t p2 = pack_bf16x2(__uint_as_float(r[8 * j + 4]) + b1.x, __uint_as_float(r[8 * j + 5]) + b1.y);
+      const uint32_t p3 = pack_bf16x2(__uint_as_float(r[8 * j + 6]) + b1.z, __uint_as_float(r[8 * j + 7]) + b1.w);
+      const uint32_t dst = row_base + (uint32_t)(((hh * 4 + j) ^ (lane & 7)) << 4);
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(p0), "r"(p1), "r"(p2), "r"(p3) : "memory");
+    }
+  }
+  __syncwarp();
+  const int chunk = lane & 7;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = (lane >> 3) + 4 * i;
+    const int dst = __shfl_sync(0xffffffffu, dst_elem, row);
+    uint32_t v0, v1, v2, v3;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3)
+                 : "r"(stage + (uint32_t)row * 128u + (uint32_t)((chunk ^ (row & 7)) << 4)) : "memory");
+    if (dst >= 0) *reinterpret_cast<uint4*>(cache + dst + chunk * 8) = make_uint4(v0, v1, v2, v3);
+  }
+  __syncwarp();                                         // the box may be refilled
 }
 
 template <int EPI> struct EpiCols { static constexpr int value = (EPI == 1) ? 32 : 64; };

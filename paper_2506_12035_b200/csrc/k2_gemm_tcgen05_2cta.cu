@@ -52,7 +52,8 @@ template <int BN, int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                          const __grid_constant__ CUtensorMap tmap_out, int M, int N, int K,
-                         const float* __restrict__ bias, int* __restrict__ status, int* __restrict__ turn) {
+                         const float* __restrict__ bias, int* __restrict__ status, int* __restrict__ turn,
+                         const KvScatter kv) {
   using Cfg = PairCfg<BN>;
   constexpr int STAGES = Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
@@ -244,10 +245,27 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
         }
         constexpr int EC = EpiCols<EPI>::value;
         const float* bias_tile = kb0 == 0 ? bias + n_blk * BN : nullptr;    // the piece with K-block 0 adds the bias
+        if (EPI == 4 && n_blk * BN >= kv.D) {
+          // a K or V tile of the fused QKV projection: straight into the cache rows of the active tokens
+          const int which = (n_blk * BN) / kv.D - 1;                        // 0 = K, 1 = V
+          const int col0 = n_blk * BN - (which + 1) * kv.D;
+          const int grow = row0 + lane;
+          int dst_row = -1;
+          if (grow < M) {
+            const int b = grow / kv.n;
+            const int t = kv.idx ? kv.idx[grow] : grow - b * kv.n;
+            dst_row = ((which * kv.B + b) * kv.S + t) * kv.D + col0;
+          }
 #pragma unroll 1
-        for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += EC)
-          epilogue_box<EPI>(t_row + (uint32_t)c0, bias_tile ? bias_tile + c0 : nullptr, &tmap_out, n_blk * BN + c0, row0,
-                            my_stage, lane);
+          for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 64)
+            epilogue_box_scatter(t_row + (uint32_t)c0, bias_tile + c0, (bf16*)kv.cache, dst_row < 0 ? -1 : dst_row + c0, my_stage,
+                                 lane);
+        } else {
+#pragma unroll 1
+          for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += EC)
+            epilogue_box<(EPI == 4) ? 0 : EPI>(t_row + (uint32_t)c0, bias_tile ? bias_tile + c0 : nullptr, &tmap_out,
+                                               n_blk * BN + c0, row0, my_stage, lane);
+        }
         if (my_turn && lane == 0) {
           if (kb0 == 0 && kb1 < n_kb) {
             ptx::bulk_wait_all();                           // this warp's reduce-adds have been performed
@@ -286,7 +304,7 @@ bool make_map_2d(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols
 
 template <int BN, int EPI>
 cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& to, int M, int N, int K,
-                        const float* bias, int* status, int* turn, cudaStream_t st) {
+                        const float* bias, int* status, int* turn, const KvScatter& kv, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_2cta_kernel<BN, EPI>,
@@ -303,7 +321,7 @@ cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUte
   int* use_turn = (EPI == 1 && turn && n_tiles > max_pairs && n_tiles % max_pairs != 0 && n_tiles < 4 * max_pairs)
                       ? turn : nullptr;
   return launch_pdl(gemm_tcgen05_2cta_kernel<BN, EPI>, dim3(2 * pairs), dim3(kThreads), (size_t)PairCfg<BN>::SMEM_BYTES,
-                    st, ta, tw, to, M, N, K, bias, status, use_turn);
+                    st, ta, tw, to, M, N, K, bias, status, use_turn, kv);
 }
 
 }  // namespace
@@ -328,8 +346,17 @@ size_t gemm_tcgen05_2cta_turn_bytes(int M, int N) {
 }
 
 cudaError_t launch_gemm_tcgen05_2cta(const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
-                                     int epilogue, void* out, int* status, cudaStream_t st, int* turn) {
+                                     int epilogue, void* out, int* status, cudaStream_t st, int* turn,
+                                     const KvScatter* kv_scatter) {
   if (M == 0) return cudaSuccess;
+  KvScatter kv = {nullptr, nullptr, 1, 1, 1, 1 << 30};
+  if (epilogue == 4) {
+    // q, K and V column ranges must each be whole tiles, and cache offsets must fit 32 bits
+    if (!kv_scatter || !kv_scatter->cache || N != 3 * kv_scatter->D || kv_scatter->D % 256 ||
+        (long)2 * kv_scatter->B * kv_scatter->S * kv_scatter->D >= (1L << 31) || ((uintptr_t)kv_scatter->cache & 15))
+      return cudaErrorInvalidValue;
+    kv = *kv_scatter;
+  }
   if (N % 128 || K % BK || lda % 8 || ((uintptr_t)a & 15) || ((uintptr_t)w & 15)) return cudaErrorInvalidValue;
   const int bn = gemm_tcgen05_2cta_pick_bn(M, N);
   CUtensorMap ta, tw, to;
@@ -338,8 +365,8 @@ cudaError_t launch_gemm_tcgen05_2cta(const void* a, int lda, int M, const void* 
   if (((uintptr_t)out & 15) || !tma_make_store_map(&to, out, (uint64_t)M, (uint64_t)N, epilogue == 1 ? 4 : 2))
     return cudaErrorInvalidValue;
 #define MARCHE_GEMM2_CASE(BN_, EPI_) \
-  if (bn == BN_ && epilogue == EPI_) return launch_pair<BN_, EPI_>(ta, tw, to, M, N, K, bias, status, turn, st);
-  MARCHE_GEMM2_CASE(256, 0) MARCHE_GEMM2_CASE(256, 1) MARCHE_GEMM2_CASE(256, 2)
+  if (bn == BN_ && epilogue == EPI_) return launch_pair<BN_, EPI_>(ta, tw, to, M, N, K, bias, status, turn, kv, st);
+  MARCHE_GEMM2_CASE(256, 0) MARCHE_GEMM2_CASE(256, 1) MARCHE_GEMM2_CASE(256, 2) MARCHE_GEMM2_CASE(256, 4)
   MARCHE_GEMM2_CASE(128, 0) MARCHE_GEMM2_CASE(128, 1) MARCHE_GEMM2_CASE(128, 2)
 #undef MARCHE_GEMM2_CASE
   return cudaErrorInvalidValue;

@@ -61,11 +61,22 @@ cudaError_t launch_gemm_simt(bool bf16_t, const void* a, int lda, int M, const v
 cudaError_t launch_gemm_tcgen05(const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
                                 int epilogue, void* out, int* status, cudaStream_t st);
 int gemm_tcgen05_pick_bn(int M, int N);
+// Where the K and V columns of a fused QKV projection go (Algorithm 1 line 11 done by the projection's
+// epilogue, epilogue code 4): row r of the GEMM is active token j = r % n of sample b = r / n, its cache row is
+// idx[r] (identity when idx is NULL).  cache is one block's [2][B][S][D] slice (bf16).  Needs N == 3 D,
+// D a multiple of 256 and 2 B S D < 2^31.
+struct KvScatter {
+  const int32_t* idx;
+  void* cache;
+  int n, S, B, D;
+};
+
 // Same contract, tcgen05.mma cta_group::2: CTA pairs share 256 x BN tiles (cluster of 2, no multicast).
 // `turn`: optional zero-filled device scratch of gemm_tcgen05_2cta_turn_bytes(M, N) bytes; with it the
 // residual epilogue may use stream-K (ordered reduce-adds; the flags are left zero again).
 cudaError_t launch_gemm_tcgen05_2cta(const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
-                                     int epilogue, void* out, int* status, cudaStream_t st, int* turn = nullptr);
+                                     int epilogue, void* out, int* status, cudaStream_t st, int* turn = nullptr,
+                                     const KvScatter* kv_scatter = nullptr);
 size_t gemm_tcgen05_2cta_turn_bytes(int M, int N);
 int gemm_tcgen05_2cta_pick_bn(int M, int N);
 
