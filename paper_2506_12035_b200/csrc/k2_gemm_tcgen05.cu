@@ -201,13 +201,9 @@ int sm_count() { return device_sm_count(); }
 template <int BN, int EPI>
 cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& to, int M, int N, int K,
                        const float* bias, int* status, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         GemmCfg<BN>::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static size_t smem_set[kMaxDevices] = {};
+  cudaError_t e = ensure_dynamic_smem(gemm_tcgen05_kernel<BN, EPI>, (size_t)GemmCfg<BN>::SMEM_BYTES, smem_set);
+  if (e != cudaSuccess) return e;
   const int n_tiles = ((M + BM - 1) / BM) * (N / BN);
   const int grid = n_tiles < sm_count() ? n_tiles : sm_count();
   return launch_pdl(gemm_tcgen05_kernel<BN, EPI>, dim3(grid), dim3(kGemmThreads), (size_t)GemmCfg<BN>::SMEM_BYTES, st, ta,

@@ -305,13 +305,9 @@ bool make_map_2d(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols
 template <int BN, int EPI>
 cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& to, int M, int N, int K,
                         const float* bias, int* status, int* turn, const KvScatter& kv, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_2cta_kernel<BN, EPI>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<BN>::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static size_t smem_set[kMaxDevices] = {};
+  cudaError_t e = ensure_dynamic_smem(gemm_tcgen05_2cta_kernel<BN, EPI>, (size_t)PairCfg<BN>::SMEM_BYTES, smem_set);
+  if (e != cudaSuccess) return e;
   const int n_tiles = ((M + 2 * BM - 1) / (2 * BM)) * (N / BN);
   const int max_pairs = device_sm_count() / 2;
   const int pairs = n_tiles < max_pairs ? n_tiles : max_pairs;

@@ -332,13 +332,9 @@ template <int DH, int NWARPS, bool SCORING>
 cudaError_t launch_att(const CUtensorMap& tm, const bf16* q, int ld_q, int B, int n, int S, int H,
                        const uint8_t* is_new, float* partial, f16* o, int* status, WriteBack wb, cudaStream_t st) {
   const size_t smem = NSTAGE * AttCfg<DH>::STAGE_BYTES + 1024 + 64 + (SCORING ? (size_t)NWARPS * S * sizeof(float) : 0);
-  static size_t smem_set = 0;
-  if (smem > smem_set) {
-    cudaError_t e = cudaFuncSetAttribute(attention_mma_kernel<DH, NWARPS, SCORING>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    smem_set = smem;
-  }
+  static size_t smem_set[kMaxDevices] = {};
+  cudaError_t e = ensure_dynamic_smem(attention_mma_kernel<DH, NWARPS, SCORING>, smem, smem_set);
+  if (e != cudaSuccess) return e;
   // (Launching one sample's heads as a cluster, to co-schedule the CTAs that read neighbouring
   // 128-byte pieces of the same cache rows, was measured and does not help: 41.0 -> 41-43 us.)
   return launch_pdl(attention_mma_kernel<DH, NWARPS, SCORING>, dim3(B * H), dim3((NWARPS + 1) * 32), smem, st, tm, q, ld_q,

@@ -93,12 +93,14 @@ cudaError_t launch_attention_simt(bool bf16_t, const void* q, int ld_q, int B, i
   const long kv_stride = (long)B * S * H * dh;
   cudaError_t e;
   if (bf16_t) {
-    e = cudaFuncSetAttribute(attention_simt_kernel<bf16, f16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static size_t smem_set[kMaxDevices] = {};
+    e = ensure_dynamic_smem(attention_simt_kernel<bf16, f16>, smem, smem_set);
     if (e != cudaSuccess) return e;
     return launch_pdl(attention_simt_kernel<bf16, f16>, dim3(B * H), dim3(kAttWarps * 32), smem, st, (const bf16*)q, ld_q,
                       n, S, H, dh, (const bf16*)cache_layer, kv_stride, is_new, score_partial, (f16*)o);
   } else {
-    e = cudaFuncSetAttribute(attention_simt_kernel<float, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static size_t smem_set[kMaxDevices] = {};
+    e = ensure_dynamic_smem(attention_simt_kernel<float, float>, smem, smem_set);
     if (e != cudaSuccess) return e;
     return launch_pdl(attention_simt_kernel<float, float>, dim3(B * H), dim3(kAttWarps * 32), smem, st, (const float*)q,
                       ld_q, n, S, H, dh, (const float*)cache_layer, kv_stride, is_new, score_partial, (float*)o);

@@ -376,13 +376,9 @@ template <bool SCORING>
 cudaError_t launch_tc(const CUtensorMap& tkv, const CUtensorMap& tq, int B, int n, int S, int H, const uint8_t* is_new,
                       float* partial, f16* o, int* status, cudaStream_t st) {
   const size_t smem = SMEM_FIXED + (SCORING ? (size_t)4 * S * sizeof(float) : 0);
-  static size_t smem_set = 0;
-  if (smem > smem_set) {
-    cudaError_t e = cudaFuncSetAttribute(attention_tcgen05_kernel<SCORING>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
-    if (e != cudaSuccess) return e;
-    smem_set = smem;
-  }
+  static size_t smem_set[kMaxDevices] = {};
+  cudaError_t e = ensure_dynamic_smem(attention_tcgen05_kernel<SCORING>, smem, smem_set);
+  if (e != cudaSuccess) return e;
   return launch_pdl(attention_tcgen05_kernel<SCORING>, dim3(B * H), dim3(kThreads), smem, st, tkv, tq, n, S, H, B, is_new,
                     partial, o, status);
 }

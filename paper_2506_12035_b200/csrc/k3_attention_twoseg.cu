@@ -342,13 +342,9 @@ cudaError_t launch_ts(const CUtensorMap& tc, const CUtensorMap& ta, const bf16* 
                       float* partial, f16* o, int* status, cudaStream_t st) {
   const size_t smem = NSTAGE * AttCfg<DH>::STAGE_BYTES + 1024 + 64 + 32 * 8 + 32 + (((size_t)n * 4 + 15) & ~(size_t)15) +
                       (SCORING ? (size_t)NWARPS * S * sizeof(float) : 0);
-  static size_t smem_set = 0;
-  if (smem > smem_set) {
-    cudaError_t e = cudaFuncSetAttribute(attention_twoseg_kernel<DH, NWARPS, SCORING>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    smem_set = smem;
-  }
+  static size_t smem_set[kMaxDevices] = {};
+  cudaError_t e = ensure_dynamic_smem(attention_twoseg_kernel<DH, NWARPS, SCORING>, smem, smem_set);
+  if (e != cudaSuccess) return e;
   return launch_pdl(attention_twoseg_kernel<DH, NWARPS, SCORING>, dim3(B * H), dim3((NWARPS + 1) * 32), smem, st, tc, ta,
                     qkv, ld, k_off, v_off, n, S, H, B, idx, cache, is_new, partial, o, status);
 }

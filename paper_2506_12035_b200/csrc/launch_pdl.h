@@ -26,6 +26,22 @@ inline bool pdl_enabled() {
   return on == 1;
 }
 
+// Raises a kernel's dynamic shared-memory limit to at least `bytes` on the current device.  The
+// attribute belongs to the device's context, so what has been set is remembered per device
+// (`cache`: one zero-initialised array per kernel instantiation at the call site).
+constexpr int kMaxDevices = 64;
+template <typename Kernel>
+cudaError_t ensure_dynamic_smem(Kernel kernel, size_t bytes, size_t (&cache)[kMaxDevices]) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (bytes <= cache[dev]) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess) cache[dev] = bytes;
+  return e;
+}
+
 // cluster_x > 1 additionally launches the grid in clusters of that many consecutive CTAs (used only
 // to co-schedule CTAs that stream neighbouring bytes of the same DRAM pages; no cluster-level
 // synchronisation or shared memory is involved).
