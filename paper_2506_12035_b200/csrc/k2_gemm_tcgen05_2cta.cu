@@ -314,8 +314,11 @@ cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUte
   // stream-K only for the reduce-add epilogue and only where whole tiles would waste a large part of
   // the last wave: a few waves at most (measured: +2 % on the cache-aware step, but -4 % on the
   // 9-wave full step, where the ordering costs more than the 4 % of idle SMs it removes)
-  int* use_turn = (EPI == 1 && turn && n_tiles > max_pairs && n_tiles % max_pairs != 0 && n_tiles < 4 * max_pairs)
-                      ? turn : nullptr;
+  // ... and only for long tiles (K >= 2048, i.e. fc2): the completing piece has to wait until the first
+  // piece's reduce-adds are complete, about 3 us after its last MMA, which a 16-K-block tile (7 us of MMA
+  // work, the out-projection) cannot hide: measured 18 us with and without stream-K there.
+  int* use_turn = (EPI == 1 && turn && K >= 2048 && n_tiles > max_pairs && n_tiles % max_pairs != 0 &&
+                   n_tiles < 4 * max_pairs) ? turn : nullptr;
   return launch_pdl(gemm_tcgen05_2cta_kernel<BN, EPI>, dim3(2 * pairs), dim3(kThreads), (size_t)PairCfg<BN>::SMEM_BYTES,
                     st, ta, tw, to, M, N, K, bias, status, use_turn, kv);
 }
