@@ -53,7 +53,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                          const __grid_constant__ CUtensorMap tmap_out, int M, int N, int K,
                          const float* __restrict__ bias, int* __restrict__ status, int* __restrict__ turn,
-                         const KvScatter kv) {
+                         const KvScatter kv, int tail_split) {
   using Cfg = PairCfg<BN>;
   constexpr int STAGES = Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
@@ -86,7 +86,11 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
   //    late; the two TMA reduce-adds into the fp32 output are ordered by a per-(tile, rank, warp) turn
   //    flag in global memory (0 -> 1 by the first piece, back to 0 by the second), which keeps the
   //    result bit-reproducible.
-  int n_pieces, sk_u0 = 0, sk_u1 = 0, sk_t_last = 0;
+  //  * tail_split > 1 (whole-tile mode only): the tiles left over after the last full round
+  //    (n_tiles mod n_pairs of them) are cut along N into tail_split column slices each, and the slices
+  //    are dealt round-robin, so the last round costs about 1/tail_split of a tile instead of a whole one.
+  //    A slice loads the same W box (only its first rows are used) and issues MMAs with N = BN / tail_split.
+  int n_pieces, sk_u0 = 0, sk_u1 = 0, sk_t_last = 0, full_rounds = 0;
   if (turn) {
     const long U = (long)n_tiles * n_kb;
     const long W = (U + n_pairs - 1) / n_pairs;
@@ -94,19 +98,33 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
     sk_u1 = (int)((long)sk_u0 + W < U ? (long)sk_u0 + W : U);
     sk_t_last = sk_u1 > sk_u0 ? (sk_u1 - 1) / n_kb : 0;
     n_pieces = sk_u1 > sk_u0 ? sk_t_last - sk_u0 / n_kb + 1 : 0;
+  } else if (tail_split > 1) {
+    full_rounds = n_tiles / n_pairs;
+    const int slices = (n_tiles - full_rounds * n_pairs) * tail_split;
+    n_pieces = full_rounds + (slices > pair ? (slices - pair + n_pairs - 1) / n_pairs : 0);
   } else {
     n_pieces = pair < n_tiles ? (n_tiles - pair + n_pairs - 1) / n_pairs : 0;
   }
-  auto get_piece = [&](int i, int& tile, int& kb0, int& kb1) {
+  // piece i of this pair: output tile, K-block range, and the column slice [n_off, n_off + n_w) of the tile
+  auto get_piece = [&](int i, int& tile, int& kb0, int& kb1, int& n_off, int& n_w) {
+    n_off = 0;
+    n_w = BN;
     if (turn) {
       tile = sk_t_last - i;
       const int lo = tile * n_kb, hi = lo + n_kb;
       kb0 = (sk_u0 > lo ? sk_u0 : lo) - lo;
       kb1 = (sk_u1 < hi ? sk_u1 : hi) - lo;
     } else {
-      tile = pair + i * n_pairs;
       kb0 = 0;
       kb1 = n_kb;
+      if (tail_split > 1 && i >= full_rounds) {
+        const int j = pair + (i - full_rounds) * n_pairs;
+        tile = full_rounds * n_pairs + j / tail_split;
+        n_w = BN / tail_split;
+        n_off = (j % tail_split) * n_w;
+      } else {
+        tile = pair + i * n_pairs;
+      }
     }
   };
 
@@ -146,9 +164,9 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       ptx::prefetch_tensormap(&tmap_out);
       int prefetched = 0;                                  // ring slots whose barrier is armed and W half loaded
       if (n_pieces > 0) {
-        int tile, kb0, kb1;
-        get_piece(0, tile, kb0, kb1);
-        const int wrow0 = (tile % n_n) * BN + (int)rank * (BN / 2);
+        int tile, kb0, kb1, n_off, n_w;
+        get_piece(0, tile, kb0, kb1, n_off, n_w);
+        const int wrow0 = (tile % n_n) * BN + n_off + (int)rank * (n_w / 2);
         for (; prefetched < STAGES && kb0 + prefetched < kb1; ++prefetched) {
           const uint32_t leader_full = ptx::mapa(full_bar(prefetched), 0);
           if (rank == 0) ptx::mbar_expect_tx(full_bar(prefetched), 2 * Cfg::STAGE_BYTES);
@@ -159,11 +177,11 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       int it = 0;
       bool ok = true;
       for (int i = 0; i < n_pieces && ok; ++i) {
-        int tile, kb0, kb1;
-        get_piece(i, tile, kb0, kb1);
+        int tile, kb0, kb1, n_off, n_w;
+        get_piece(i, tile, kb0, kb1, n_off, n_w);
         const int m2 = tile / n_n, n_blk = tile - m2 * n_n;
         const int row0 = m2 * 2 * BM + (int)rank * BM;                // this CTA's 128 rows of A
-        const int wrow0 = n_blk * BN + (int)rank * (BN / 2);          // this CTA's half of the W tile
+        const int wrow0 = n_blk * BN + n_off + (int)rank * (n_w / 2);  // this CTA's half of the W rows of the slice
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t leader_full = ptx::mapa(full_bar(s), 0);
@@ -183,12 +201,12 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer (leader only)
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = ptx::idesc_f16_f32(2 * BM, BN);
       int it = 0;
       bool ok = true;
       for (int i = 0; i < n_pieces && ok; ++i) {
-        int tile, kb0, kb1;
-        get_piece(i, tile, kb0, kb1);
+        int tile, kb0, kb1, n_off, n_w;
+        get_piece(i, tile, kb0, kb1, n_off, n_w);
+        const uint32_t idesc = ptx::idesc_f16_f32(2 * BM, n_w);
         const int acc = i & 1;
         const uint32_t acc_ph = (uint32_t)(i >> 1) & 1u;
         if (!ptx::mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -217,8 +235,8 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
     const int half = (warp - 2) >> 2;                       // which half of the BN columns
     bool ok = true;
     for (int i = 0; i < n_pieces && ok; ++i) {
-      int tile, kb0, kb1;
-      get_piece(i, tile, kb0, kb1);
+      int tile, kb0, kb1, n_off, n_w;
+      get_piece(i, tile, kb0, kb1, n_off, n_w);
       const int m2 = tile / n_n, n_blk = tile - m2 * n_n;
       const int acc = i & 1;
       const uint32_t acc_ph = (uint32_t)(i >> 1) & 1u;
@@ -244,11 +262,16 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
           if (*abort_flag) { ok = false; break; }
         }
         constexpr int EC = EpiCols<EPI>::value;
-        const float* bias_tile = kb0 == 0 ? bias + n_blk * BN : nullptr;    // the piece with K-block 0 adds the bias
-        if (EPI == 4 && n_blk * BN >= kv.D) {
+        const int col_tile = n_blk * BN + n_off;                            // first output column of this piece
+        const float* bias_tile = kb0 == 0 ? bias + col_tile : nullptr;     // the piece with K-block 0 adds the bias
+        // the two warps of a TMEM lane quarter share the piece's n_w columns (a 64-column slice of a
+        // 64-column-box epilogue is handled by the first of them alone)
+        const int hw = n_w / 2 > EC ? n_w / 2 : EC;
+        const int c_begin = half * hw, c_end = (half + 1) * hw < n_w ? (half + 1) * hw : n_w;
+        if (EPI == 4 && col_tile >= kv.D) {
           // a K or V tile of the fused QKV projection: straight into the cache rows of the active tokens
-          const int which = (n_blk * BN) / kv.D - 1;                        // 0 = K, 1 = V
-          const int col0 = n_blk * BN - (which + 1) * kv.D;
+          const int which = col_tile / kv.D - 1;                            // 0 = K, 1 = V
+          const int col0 = col_tile - (which + 1) * kv.D;
           const int grow = row0 + lane;
           int dst_row = -1;
           if (grow < M) {
@@ -257,14 +280,14 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
             dst_row = ((which * kv.B + b) * kv.S + t) * kv.D + col0;
           }
 #pragma unroll 1
-          for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 64)
-            epilogue_box_scatter(t_row + (uint32_t)c0, bias_tile + c0, (bf16*)kv.cache, dst_row < 0 ? -1 : dst_row + c0, my_stage,
-                                 lane);
+          for (int c0 = c_begin; c0 < c_end; c0 += 64)
+            epilogue_box_scatter(t_row + (uint32_t)c0, bias_tile + c0, (bf16*)kv.cache, dst_row < 0 ? -1 : dst_row + c0,
+                                 my_stage, lane);
         } else {
 #pragma unroll 1
-          for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += EC)
+          for (int c0 = c_begin; c0 < c_end; c0 += EC)
             epilogue_box<(EPI == 4) ? 0 : EPI>(t_row + (uint32_t)c0, bias_tile ? bias_tile + c0 : nullptr, &tmap_out,
-                                               n_blk * BN + c0, row0, my_stage, lane);
+                                               col_tile + c0, row0, my_stage, lane);
         }
         if (my_turn && lane == 0) {
           if (kb0 == 0 && kb1 < n_kb) {
@@ -319,8 +342,25 @@ cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUte
   // work, the out-projection) cannot hide: measured 18 us with and without stream-K there.
   int* use_turn = (EPI == 1 && turn && K >= 2048 && n_tiles > max_pairs && n_tiles % max_pairs != 0 &&
                    n_tiles < 4 * max_pairs) ? turn : nullptr;
+  // Whole-tile mode: cut the tiles of the last, partial round into 2 or 4 column slices when that
+  // shortens the round (cost model in tile units: a slice costs its share of the tile plus about 0.12
+  // for its own ramp and epilogue).  MARCHE_TAIL_SPLIT=0 turns it off.
+  static int split_on = -1;
+  if (split_on < 0) {
+    const char* e = getenv("MARCHE_TAIL_SPLIT");
+    split_on = (e && e[0] == '0') ? 0 : 1;
+  }
+  int tail_split = 1;
+  const int left = n_tiles % pairs;
+  if (!use_turn && split_on && BN == 256 && left > 0) {
+    double best = 1.0;
+    for (int sp = 2; sp <= 4; sp *= 2) {
+      const double cost = (double)((left * sp + pairs - 1) / pairs) * (1.0 / sp + 0.12);
+      if (cost < best - 0.05) { best = cost; tail_split = sp; }
+    }
+  }
   return launch_pdl(gemm_tcgen05_2cta_kernel<BN, EPI>, dim3(2 * pairs), dim3(kThreads), (size_t)PairCfg<BN>::SMEM_BYTES,
-                    st, ta, tw, to, M, N, K, bias, status, use_turn, kv);
+                    st, ta, tw, to, M, N, K, bias, status, use_turn, kv, tail_split);
 }
 
 }  // namespace

@@ -328,3 +328,32 @@ def test_validate_indices():
         with pytest.raises(MarcheError) as e:
             m.validate_indices(idx_dev(bad_act), idx_dev(bad_new), None if bad_excl is None else idx_dev(bad_excl))
         assert e.value.code == -5
+
+
+@pytest.mark.parametrize("M,N,K", [(4800, 1024, 256), (9000, 768, 128), (5248, 3072, 192), (19100, 256, 128)])
+def test_linear_many_tiles_all_epilogues(M, N, K):
+    """Shapes with more output tiles than CTA pairs and a partial last round, where the pair GEMM
+    cuts the left-over tiles into column slices (and, for the residual epilogue with long K, uses
+    stream-K): every element against the oracle's product."""
+    dtype = "bf16"
+    cfg, blocks, m = model_for(dtype, 256, 4, 1024, 68, 2)
+    rng = np.random.default_rng(M + N + K)
+    a = rng.standard_normal((M, K)).astype(np.float32)
+    w = (rng.standard_normal((N, K)) * 0.05).astype(np.float32)
+    bias = rng.standard_normal(N).astype(np.float32)
+    aq, wq = quant_a(a, dtype), quant_a(w, dtype)
+    acc = orc.linear(aq, wq, bias.astype(np.float64))
+    a_d, w_d, b_d = dev(a, adt(dtype)), dev(w, adt(dtype)), dev(bias)
+    out = torch.zeros(M + 3, N, dtype=tdt(dtype), device="cuda")
+    m.linear(a_d, w_d, b_d, 0, out, M=M)
+    assert max_abs(host(out[:M]), acc) <= 3e-2 and rel_l2(host(out[:M]), acc) <= 4e-3
+    assert (host(out[M:]) == 0).all()                                    # rows beyond M untouched
+    res = rng.standard_normal((M, N)).astype(np.float32)
+    out = dev(res)
+    m.linear(a_d, w_d, b_d, 1, out)
+    assert max_abs(host(out), acc + res) <= 1e-4 * max(1.0, math.sqrt(K / 256))
+    out = torch.zeros(M, N, dtype=adt(dtype), device="cuda")
+    m.linear(a_d, w_d, b_d, 2, out)
+    want = orc.gelu(acc)
+    assert max_abs(host(out), want) <= 3e-2 and rel_l2(host(out), want) <= 4e-3
+    assert m.device_status() == 0
