@@ -236,6 +236,8 @@ def run_reference(args, cfg):
     if rank != 0:
         return
     vals = []
+    for _ in range(args.warmup):                 # untimed: pages in NumPy / BLAS threads and the weight generator
+        oracle_sample(cfg, args.ratio, n_cache_steps=1)
     for _ in range(args.steps):
         ips, t_gen, info = oracle_sample(cfg, args.ratio)
         vals.append((ips, t_gen))
