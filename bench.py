@@ -40,7 +40,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM traffic per launch of the dominant kernel classes from the committed ncu captures
 # (profiles/), bytes; None where no capture exists.
-NCU_TRAFFIC = {"gemm": 31.1e6,        # profiles/gemm_tcgen05_2cta_mar_l_rows4352.md (mean of the block's four GEMMs)
+NCU_TRAFFIC = {"gemm": 31.3e6,        # profiles/gemm_tcgen05_2cta_mar_l_rows4352.md (mean of the block's four GEMMs)
                "attention": 183.6e6}  # profiles/attention_mma_mar_l_nA34.md
 
 
