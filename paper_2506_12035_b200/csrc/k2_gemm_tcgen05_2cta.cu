@@ -343,19 +343,22 @@ cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUte
   int* use_turn = (EPI == 1 && turn && K >= 2048 && n_tiles > max_pairs && n_tiles % max_pairs != 0 &&
                    n_tiles < 4 * max_pairs) ? turn : nullptr;
   // Whole-tile mode: cut the tiles of the last, partial round into 2 or 4 column slices when that
-  // shortens the round (cost model in tile units: a slice costs its share of the tile plus about 0.12
-  // for its own ramp and epilogue).  MARCHE_TAIL_SPLIT=0 turns it off.
+  // shortens the round (cost model in tile units, below).  MARCHE_TAIL_SPLIT=0 turns it off.
   static int split_on = -1;
   if (split_on < 0) {
     const char* e = getenv("MARCHE_TAIL_SPLIT");
-    split_on = (e && e[0] == '0') ? 0 : 1;
+    split_on = e ? atoi(e) : 1;                      // 0 off, 1 cost model, 2 / 4 forced (measurement only)
   }
   int tail_split = 1;
   const int left = n_tiles % pairs;
-  if (!use_turn && split_on && BN == 256 && left > 0) {
+  if (!use_turn && (split_on == 2 || split_on == 4) && BN == 256 && left > 0) {
+    tail_split = split_on;
+  } else if (!use_turn && split_on && BN == 256 && left > 0) {
     double best = 1.0;
     for (int sp = 2; sp <= 4; sp *= 2) {
-      const double cost = (double)((left * sp + pairs - 1) / pairs) * (1.0 / sp + 0.12);
+      // measured at K = 1024: a half-width slice costs about 0.75 of a tile, a quarter-width one about 0.65
+      // (every slice loads the whole A tile again and pays its own ramp and epilogue)
+      const double cost = (double)((left * sp + pairs - 1) / pairs) * (1.0 / sp + (sp == 2 ? 0.25 : 0.40));
       if (cost < best - 0.05) { best = cost; tail_split = sp; }
     }
   }
