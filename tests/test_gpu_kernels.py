@@ -357,3 +357,74 @@ def test_linear_many_tiles_all_epilogues(M, N, K):
     want = orc.gelu(acc)
     assert max_abs(host(out), want) <= 3e-2 and rel_l2(host(out), want) <= 4e-3
     assert m.device_status() == 0
+
+
+@pytest.mark.parametrize("D,F", [(768, 3072), (1024, 4096), (1280, 5120)])
+@pytest.mark.parametrize("M", [256, 4352, 5760, 10176])
+def test_projection_shapes_of_the_configs(D, F, M):
+    """The four projections of a block at the row counts of the benchmark configurations (K = 1280 and
+    5120 loop counts included); 384 sampled rows of each output against the oracle's product."""
+    dtype = "bf16"
+    cfg, blocks, m = model_for(dtype, 256, 4, 1024, 68, 2)
+    rng = np.random.default_rng(D + M)
+    rows = np.unique(np.concatenate([[0, M - 1], rng.integers(0, M, 382)]))
+    for (N, K, epi) in ((3 * D, D, 0), (D, D, 1), (F, D, 2), (D, F, 1)):
+        a = rng.standard_normal((M, K)).astype(np.float32)
+        w = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+        bias = (rng.standard_normal(N) * 0.02).astype(np.float32)
+        acc = orc.linear(quant_a(a[rows], dtype), quant_a(w, dtype), bias.astype(np.float64))
+        a_d, w_d, b_d = dev(a, adt(dtype)), dev(w, adt(dtype)), dev(bias)
+        if epi == 0:
+            out = torch.zeros(M, N, dtype=tdt(dtype), device="cuda")
+            want = acc
+        elif epi == 1:
+            res = rng.standard_normal((M, N)).astype(np.float32)
+            out = dev(res)
+            want = acc + res[rows]
+        else:
+            out = torch.zeros(M, N, dtype=adt(dtype), device="cuda")
+            want = orc.gelu(acc)
+        m.linear(a_d, w_d, b_d, epi, out)
+        got = host(out)[rows]
+        lim = 1e-4 * max(1.0, math.sqrt(K / 256)) if epi == 1 else 3e-2
+        assert max_abs(got, want) <= lim, (N, K, epi, max_abs(got, want))
+        if epi != 1:
+            assert rel_l2(got, want) <= 4e-3
+    assert m.device_status() == 0
+
+
+@pytest.mark.parametrize("S", [320, 1088])
+@pytest.mark.parametrize("dh,H", [(64, 4), (80, 8)])
+@pytest.mark.parametrize("n,nG", [(159, 25), (320, 320), (97, 1)])
+def test_attention_many_rows(S, dh, H, n, nG):
+    """Active sets beyond one query tile (both tensor-core kernels are reached: tcgen05 for head_dim 64,
+    mma.sync with seven consumer warps for head_dim 80), every query scoring in one case."""
+    dtype = "bf16"
+    B, D = 2, dh * H
+    cfg, blocks, m = model_for(dtype, D, H, 128, S, B)
+    rng = np.random.default_rng(S + n + dh)
+    q = (rng.standard_normal((B * n, 3 * D)) * 3.0).astype(np.float32)
+    cache = rng.standard_normal((2, B, S, D)).astype(np.float32)
+    flags = np.zeros((B, n), dtype=np.uint8)
+    for b in range(B):
+        flags[b, rng.permutation(n)[:nG]] = 1
+    o = torch.zeros(B * n, D, dtype=adt(dtype), device="cuda")
+    partial = torch.full((B, H, S), -1.0, device="cuda")
+    m.attention(dev(q, tdt(dtype)), 3 * D, n, dev(cache, tdt(dtype)), dev(flags), partial, o)
+    qq, cc = quant(q, dtype), quant(cache, dtype)
+    want_o = np.zeros((B * n, D))
+    want_p = np.zeros((B, H, S))
+    for b in range(B):
+        for h in range(H):
+            c = slice(h * dh, (h + 1) * dh)
+            z, p = orc.softmax_attention(qq[b * n:(b + 1) * n, c], cc[0, b][:, c], cc[1, b][:, c])
+            want_o[b * n:(b + 1) * n, c] = z
+            want_p[b, h] = p[flags[b].astype(bool)].sum(axis=0)
+    got_o, got_p = host(o), host(partial)
+    assert rel_l2(got_o, want_o) <= 8e-3 and max_abs(got_o, want_o) <= 3e-2
+    assert max_abs(got_p, want_p) <= 2e-2 * max(1, nG) / 8 + 1e-6
+    assert np.allclose(got_p.sum(-1), nG, rtol=5e-3, atol=1e-6)
+    o2 = torch.zeros_like(o)
+    m.attention(dev(q, tdt(dtype)), 3 * D, n, dev(cache, tdt(dtype)), None, None, o2)       # plain flavour
+    assert rel_l2(host(o2), want_o) <= 8e-3 and max_abs(host(o2), want_o) <= 3e-2
+    assert m.device_status() == 0
