@@ -46,7 +46,7 @@ struct WriteBack {
 
 // NWARPS consumer warps (16 query rows each) plus one producer warp.
 template <int DH, int NWARPS, bool SCORING>
-__global__ void __launch_bounds__((NWARPS + 1) * 32)
+__global__ void __launch_bounds__((NWARPS + 1) * 32, NWARPS == 3 ? 4 : 1)
 attention_mma_kernel(const __grid_constant__ CUtensorMap tmap_kv, const bf16* __restrict__ q, int ld_q, int n,
                      int S, int H, int B, const uint8_t* __restrict__ is_new, float* __restrict__ score_partial,
                      f16* __restrict__ o, int* __restrict__ status, WriteBack wb) {
