@@ -354,6 +354,20 @@ def run_ours(args, cfg):
                             "peak_source": "%s (%s)" % (peak_kind, "sustained bf16 GEMM" if dom["bound"] == "tensor" else "device copy"),
                             "timing": "CUDA events in front of every launch, cache-aware steps of one generation of the timed workload"}
 
+        # ---- the same generation captured once in a CUDA graph and replayed (no host launch cost at all)
+        if n_dec is None:
+            try:
+                l0 = m.launch_count()
+                graph = gen.capture(hidden0)
+                per_replay = (m.launch_count() - l0) // 2          # one eager generation, one recorded
+                graph.replay()
+                ms_graph = timed(lambda: graph.replay(), 2)
+                line["cuda_graph"] = {"value": world * n_images / (ms_graph * 1e-3), "unit": "images/s",
+                                      "ms_per_step": ms_graph, "kernel_nodes_per_replay": int(per_replay)}
+                assert m.device_status() == 0
+            except Exception as exc:                      # capture is an extra; the stream path is the benchmark
+                line["cuda_graph"] = {"unavailable": str(exc)[:200]}
+
         # ---- per-step latency: events between the steps of one more generation
         if n_dec is None:
             evs = [torch.cuda.Event(enable_timing=True) for _ in range(cfg.T + 1)]

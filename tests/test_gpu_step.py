@@ -418,3 +418,21 @@ def test_maximum_sizes(shape):
     out = torch.empty(cfg.B, rd.shape[1], dtype=torch.int32, device="cuda")
     m.select_refresh(dev(so), idx_dev(G), None, rd.shape[1], out, mask)
     assert np.array_equal(out.cpu().numpy(), ro)
+
+
+def test_generation_replayed_from_a_cuda_graph():
+    """A generation recorded in a CUDA graph writes the same bytes as the eager one."""
+    cfg = CASES["marb_slice"]
+    blocks = synth.make_weights(cfg)
+    hidden0 = dev(synth.make_hidden(cfg))
+    sets = synth.new_token_sets(cfg, synth.generation_orders(cfg))
+    m, gen = gpu_generation(cfg, blocks, sets, cfg.ratio)
+    gen.run(hidden0)
+    torch.cuda.synchronize()
+    want_out, want_cache = gen.hidden_out.clone(), gen.cache.clone()
+    graph = gen.capture(hidden0)
+    gen.hidden_out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert m.device_status() == 0
+    assert torch.equal(gen.hidden_out, want_out) and torch.equal(gen.cache, want_cache)
