@@ -60,6 +60,10 @@ class Generation:
                 m.build_active(G, self.new_sets[t - 1], R_in, k_prev, active, stream)
                 k = m.step(self.hidden, self.cache, active, G, X, self.ratio, self.hidden_out, R_out, self.workspace,
                            stream)
+            own = None
+            if record:                      # the step's own selection, before any forcing
+                torch.cuda.synchronize()
+                own = R_out[: B * k].view(B, k).cpu().numpy().copy()
             if forced_refresh is not None:
                 fr = forced_refresh[t]
                 k = fr.shape[1]
@@ -68,7 +72,7 @@ class Generation:
                 m.get_scores(self.workspace, self.scores, stream)
                 torch.cuda.synchronize()
                 log.append(dict(
-                    t=t, n_active=n_active,
+                    t=t, n_active=n_active, refresh_own=own,
                     active=None if (t == 0 or mode == "full") else active.cpu().numpy().copy(),
                     scores=self.scores.cpu().numpy().copy(),
                     refresh=R_out[: B * k].view(B, k).cpu().numpy().copy(),

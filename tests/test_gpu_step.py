@@ -66,8 +66,14 @@ def test_teacher_forced_generation(case, ratio):
         unit = cfg.H * nG / cfg.S                                      # mean score
         assert max_abs(g["scores"], rec["scores"]) <= (5e-2 if cfg.dtype == "bf16" else 1e-4) * unit
         assert np.allclose(g["scores"].sum(-1), cfg.H * nG, rtol=1e-3)
-        # selection: fed the oracle's fp32 scores, the device's top-k is bit-exact
+        # the step's own selection (head-partial reduction + top-K at the end of the step), taken before
+        # the teacher forcing: bit-exact against the oracle's selection on the device's own scores
         k = rec["refresh"].shape[1]
+        assert g["refresh_own"].shape == (cfg.B, k)
+        if k:
+            assert np.array_equal(g["refresh_own"],
+                                  orc.select_refresh(g["scores"], rec["new"], rec["exclude"] if rec["exclude"].shape[1] else None, k))
+        # selection: fed the oracle's fp32 scores, the device's top-k is bit-exact
         if k:
             out = torch.empty(cfg.B, k, dtype=torch.int32, device="cuda")
             excl = rec["exclude"]
@@ -148,6 +154,44 @@ def test_invariants_untouched_rows_full_equivalence_reproducibility(dtype):
         res.append((o3.clone(), c3, s3, r3.clone()))
     for x, y in zip(*res):
         assert torch.equal(x, y)
+
+
+@pytest.mark.parametrize("B,nA", [(8, 41), (16, 45), (4, 27)])
+def test_untouched_cache_rows_byte_identical_under_fused_write_back(B, nA):
+    """Rows outside the active set keep their bytes (Algorithm 1 line 11 touches only rows of A) on the
+    production path, where the QKV projection's epilogue writes K and V straight into the cache (more than
+    128 rows: 328 and 720, the latter with a ragged last row tile); 108 rows take the separate write-back
+    kernel.  Every cache layer and hidden_out are compared byte for byte; the active rows must change."""
+    cfg = synth.CONFIGS["mar_b"].replace(L=3, E=1, B=B, T=6)
+    blocks = synth.make_weights(cfg)
+    m = make_model(cfg, blocks)
+    rng = np.random.default_rng(B)
+    S, D = cfg.S, cfg.D
+    hidden = dev(synth.make_hidden(cfg))
+    cache = m.alloc_cache()
+    ws = m.alloc_workspace(S)
+    m.init_cache(cache)
+    out = torch.zeros(B, S, D, device="cuda")
+    refresh = torch.zeros(B, S, dtype=torch.int32, device="cuda")
+    A = np.stack([rng.permutation(S)[:nA] for _ in range(B)]).astype(np.int32)
+    G = A[:, :5]
+    m.full_step(hidden, cache, idx_dev(G), None, 0.1, out, refresh, ws)
+    torch.cuda.synchronize()
+    before = cache.clone()
+    hidden2 = hidden.clone()
+    for b in range(B):
+        hidden2[b, torch.as_tensor(A[b], dtype=torch.long)] = torch.randn(nA, D, device="cuda")
+    out2 = torch.full((B, S, D), 777.0, device="cuda")
+    m.step(hidden2, cache, idx_dev(A), idx_dev(G), None, 0.1, out2, refresh, ws)
+    torch.cuda.synchronize()
+    assert m.device_status() == 0
+    for b in range(B):
+        rest = torch.as_tensor(np.setdiff1d(np.arange(S), A[b]), dtype=torch.long)
+        act = torch.as_tensor(A[b], dtype=torch.long)
+        assert torch.equal(cache[:, :, b, rest].view(torch.int16), before[:, :, b, rest].view(torch.int16))
+        changed = (cache[:, :, b, act].view(torch.int16) != before[:, :, b, act].view(torch.int16)).any(-1)
+        assert bool(changed.all())                      # every active row of every layer, K and V, was rewritten
+        assert (out2[b, rest] == 777.0).all() and (out2[b, act] != 777.0).all()
 
 
 def test_full_ratio_equals_full_recompute():

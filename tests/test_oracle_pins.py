@@ -466,6 +466,41 @@ def test_selection_ablation_policies():
     assert orc._mix32(0, 0, 0) == 0 and orc._mix32(1, 2, 3) == orc._mix32(1, 2, 3) and orc._mix32(1, 2, 3) != orc._mix32(1, 3, 2)
 
 
+def test_random_policy_hash_golden_values_and_inverse():
+    """Pins the hash of the random-selection ablation (Section 5.3) to something other than itself:
+    (i) two values derived long-hand from the formula printed in include/marche.h, stored with every
+    intermediate in tests/golden/random_policy_hash.txt; (ii) the mixing steps are a bijection on 32-bit
+    words, so undoing them - xor-shifts unwound, multipliers replaced by their inverses modulo 2^32,
+    which are computed here from the header's constants by modular inversion - must return the input
+    word; a wrong multiplier, shift amount or step order in the oracle fails one of the two."""
+    here = os.path.dirname(os.path.abspath(__file__))
+    rows = [ln.split() for ln in open(os.path.join(here, "golden", "random_policy_hash.txt"))
+            if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 2
+    for seed, b, t, want in rows:
+        assert orc._mix32(int(seed, 16), int(b, 16), int(t, 16)) == int(want, 16)
+
+    M = (1 << 32) - 1
+    inv1, inv2 = pow(0x7FEB352D, -1, 1 << 32), pow(0x846CA68B, -1, 1 << 32)
+
+    def unshift(y, s):                      # inverse of x ^= x >> s on 32 bits
+        x = y
+        for _ in range(32 // s + 1):
+            x = y ^ (x >> s)
+        return x
+
+    rng = np.random.default_rng(3)
+    for _ in range(200):
+        seed, b, t = (int(v) for v in rng.integers(0, 1 << 32, 3))
+        b, t = b % 4096, t % 2048
+        x = unshift(orc._mix32(seed, b, t), 16)
+        x = (x * inv2) & M
+        x = unshift(x, 15)
+        x = (x * inv1) & M
+        x = unshift(x, 16)
+        assert x == (seed ^ (b * 0x9E3779B1) ^ (t * 0x85EBCA77)) & M
+
+
 def test_topk_signed_zero_and_errors():
     sc = np.array([[0.0, -0.0, 0.0, -0.0]], dtype=np.float32)
     assert orc.select_refresh(sc, np.zeros((1, 0), np.int32), None, 2).tolist() == [[0, 1]]

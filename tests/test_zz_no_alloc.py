@@ -58,3 +58,21 @@ def test_static_scratch_rejects_shapes_beyond_its_size():
     assert e.value.code == -3 and "288000" in str(e.value) and "262144" in str(e.value)
     torch.cuda.synchronize()
     assert (out == -7).all()                          # nothing was enqueued
+
+
+def test_static_scratch_accepts_the_largest_shape_it_holds():
+    B, S = 128, 2048                                  # exactly 262144 bytes of mask: the limit itself
+    m = _model(B, S)
+    rng = np.random.default_rng(7)
+    scores = rng.integers(0, 50, (B, S)).astype(np.float32)
+    perm = np.stack([rng.permutation(S)[:9] for _ in range(B)]).astype(np.int32)
+    new, excl = torch.as_tensor(perm[:, :4]).cuda().contiguous(), torch.as_tensor(perm[:, 4:]).cuda().contiguous()
+    sc = torch.as_tensor(scores).cuda()
+    k = 205
+    want = torch.full((B, k), -1, dtype=torch.int32, device="cuda")
+    got = torch.full((B, k), -2, dtype=torch.int32, device="cuda")
+    m.select_refresh(sc, new, excl, k, want, torch.empty(B * S, dtype=torch.uint8, device="cuda"))
+    m.select_refresh_static(sc, new, excl, k, got)
+    torch.cuda.synchronize()
+    assert torch.equal(got, want)
+    assert np.array_equal(got.cpu().numpy(), orc.select_refresh(scores, perm[:, :4], perm[:, 4:], k))
