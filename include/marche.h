@@ -6,8 +6,11 @@
  * Conventions that hold for every call unless a call says otherwise
  * -----------------------------------------------------------------
  * Pointers   "device" pointers address global memory of the GPU that was current
- *            when marche_create() ran; "host" pointers address ordinary host
- *            memory.  The library never allocates or frees device memory: the
+ *            when marche_create() ran, and that GPU must be the current device in
+ *            every later call on the context (MARCHE_EINVAL otherwise, nothing
+ *            enqueued); "host" pointers address ordinary host memory.  Device
+ *            arrays start on 16-byte boundaries (cudaMalloc gives 256).
+ *            The library never allocates or frees device memory: the
  *            caller owns hidden states, the K/V cache, index arrays, weights
  *            and the workspace, and keeps them alive until the stream has
  *            finished the call.  The library owns only the small host-side
@@ -19,17 +22,23 @@
  *            F MLP width, L blocks, nA active tokens per sample, nG generating
  *            ("new") tokens per sample, M = B*nA rows.
  * Types      marche_config.dtype selects two element types.  `T` (q/k/v and the
- *            K/V cache, i.e. everything attention reads) is float or bf16.  `A`
- *            (both operands of the four projections: the weight matrices, and the
- *            activation matrices that feed them - LayerNorm output, attention
- *            output, GELU output) is float, or IEEE fp16 in MARCHE_BF16 contexts:
- *            with 16-bit operands the rounding of exactly these activations
- *            dominates the end-to-end error (bf16 there gives max-abs 5e-2 at 32
- *            blocks, above the 3e-2 bound; fp16 gives 7e-3), fp16 runs at the same
- *            tensor-core rate and size, and the tensor core wants both operands
- *            of one MMA in the same format.  |values| of A must stay below 65504
- *            (N(0, 0.02) weights, LayerNorm outputs, convex combinations of V rows
- *            and GELU outputs of normalised inputs do).
+ *            K/V cache, i.e. everything attention reads) and `A` (both operands of
+ *            the four projections: the weight matrices, and the activation
+ *            matrices that feed them - LayerNorm, attention and GELU outputs):
+ *              MARCHE_F32         T = A = float   (plain fp32 kernels, no tensor cores)
+ *              MARCHE_BF16        T = A = bf16    (fp32 accumulation everywhere)
+ *              MARCHE_BF16_F16OP  T = bf16, A = IEEE fp16: the weight matrices are
+ *                                 handed over in fp16
+ *            Why the third exists: with 16-bit operands the rounding of exactly the
+ *            A activations dominates the end-to-end error (all-bf16 gives max-abs
+ *            about 5e-2 against an fp64 reference at 32 blocks; fp16 there gives
+ *            under 1e-2), fp16 runs at the same tensor-core rate and size, and the
+ *            tensor core wants both operands of one MMA in the same format.
+ *            Range rule of MARCHE_BF16_F16OP: every A activation is converted with
+ *            saturation, so a magnitude above 65504 is stored as +-65504, never as
+ *            infinity (NaN stays NaN); weight matrices must already be finite fp16.
+ *            Contexts with 16-bit types have no fp32 fall-back path: a misaligned
+ *            operand is MARCHE_EINVAL, not a slower kernel.
  * Index sets int32, device, row-major [B][n] with the same n for every sample;
  *            entries are token positions in [0, S), unique within a sample.
  * Layouts    hidden / hidden_out  float [B][S][D]
@@ -59,7 +68,7 @@ extern "C" {
 typedef struct marche_ctx marche_ctx;
 typedef void* marche_stream; /* cudaStream_t */
 
-enum { MARCHE_F32 = 0, MARCHE_BF16 = 1 };
+enum { MARCHE_F32 = 0, MARCHE_BF16 = 1, MARCHE_BF16_F16OP = 2 };
 
 enum {
   MARCHE_OK = 0,
@@ -97,7 +106,7 @@ typedef struct {
   int32_t seq_len;      /* S = image tokens + buffer tokens, <= 2048                      */
   int32_t n_buffer;     /* informational (buffer tokens are ordinary tokens here)         */
   int32_t batch;        /* B, already doubled for classifier-free guidance                */
-  int32_t dtype;        /* MARCHE_F32 or MARCHE_BF16: GEMM/attention operands and cache   */
+  int32_t dtype;        /* MARCHE_F32, MARCHE_BF16 or MARCHE_BF16_F16OP (see Types above) */
   int32_t score_layer;  /* 0-based block whose attention yields the relevance scores;
                            -1 selects the second decoder block, E+1 (Section 4.2)         */
   float ln_eps;         /* LayerNorm epsilon; <= 0 selects 1e-6                           */
@@ -119,7 +128,10 @@ typedef struct {
 
 /* Creates the host-side context for one model shape on the current device.
  * `blocks` is a host array of cfg->n_blocks structs (copied).  Synchronous; no
- * device memory is allocated.  MARCHE_ESHAPE for unsupported dimensions. */
+ * device memory is allocated.  MARCHE_ESHAPE for unsupported dimensions, MARCHE_EINVAL for a
+ * NULL or misaligned parameter array.  Weight matrices and biases must be complete in memory
+ * before any call that uses them is enqueued (the projection kernels start fetching weight tiles
+ * before they wait for the preceding kernel of the stream). */
 int marche_create(const marche_config* cfg, const marche_block_weights* blocks, marche_ctx** out);
 void marche_destroy(marche_ctx* ctx);
 
@@ -389,7 +401,10 @@ int marche_gather_layernorm(marche_ctx* ctx, const float* src, int src_rows, con
 /* out = epilogue(a * w^T + bias): a A [M][K] with row stride lda elements,
  * w A [N][K], bias float [N], out [M][N] dense (type per epilogue).  The QKV,
  * output and MLP projections on active rows only (Algorithm 1 lines 5 and 9).
- * bf16: K % 64 == 0, N % 128 == 0, lda % 8 == 0.  fp32 accumulation. */
+ * 16-bit contexts: K % 64 == 0, N % 128 == 0, lda % 8 == 0 (MARCHE_ESHAPE), 16-byte aligned a, w,
+ * out (MARCHE_EINVAL).  fp32 accumulation.  w and bias must be complete in memory before the call
+ * is enqueued: synchronise after writing them, or keep at least one other kernel of the same
+ * stream between the write and this call. */
 int marche_linear(marche_ctx* ctx, const void* a, int lda, int M, const void* w, const float* bias,
                   int N, int K, int epilogue, void* out, marche_stream stream);
 
@@ -421,10 +436,32 @@ int marche_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void
  *   cache_layer i/o T [2][B][S][D]: rows outside active_idx are read, rows active_idx are written
  *   is_new / score_partial / o  as for marche_attention
  * Results equal marche_scatter_kv followed by marche_attention.  MARCHE_BF16 contexts only
- * (MARCHE_ESHAPE otherwise).  MARCHE_ATTN=twoseg makes the step use this kernel. */
+ * (MARCHE_ESHAPE otherwise).  marche_tuning.two_segment_attention makes the step use this kernel. */
 int marche_attention_two_segment(marche_ctx* ctx, const void* qkv, int ld, int n, const int32_t* active_idx,
                                  void* cache_layer, const uint8_t* is_new, float* score_partial, void* o,
                                  marche_stream stream);
+
+/* ---------------------------------------------------------------- tuning
+ * Kernel-selection switches of one context.  The defaults (marche_get_tuning after marche_create)
+ * are the measured winners on B200; the alternatives exist for measurements and for the tests that
+ * pin them to the same results.  None of them changes what is computed, only which kernel does it;
+ * `pdl` is process-wide (it is a property of how kernels are launched). */
+enum { MARCHE_ATTENTION_AUTO = 0, MARCHE_ATTENTION_MMA = 1, MARCHE_ATTENTION_TCGEN05 = 2 };
+enum { MARCHE_GEMM_AUTO = 0, MARCHE_GEMM_SINGLE = 1, MARCHE_GEMM_PAIR = 2 };
+typedef struct {
+  int32_t stream_k;              /* 1: fc2-sized residual projections use stream-K with ordered reduce-adds   */
+  int32_t fuse_qkv_scatter;      /* 1: the QKV projection's epilogue writes K, V into the cache (no K5 launch)*/
+  int32_t attention_kernel;      /* MARCHE_ATTENTION_*: AUTO picks by active rows and head_dim                 */
+  int32_t attention_tc_min_rows; /* AUTO: tcgen05 attention above this many active rows (head_dim 64)          */
+  int32_t two_segment_attention; /* 1: the step uses marche_attention_two_segment instead of K5 + K3           */
+  int32_t gemm_kernel;           /* MARCHE_GEMM_*: AUTO = CTA-pair kernel above 128 rows                       */
+  int32_t tail_split;            /* 0 off, 1 cost model, 2 / 4 forced: column slices in a partial last round   */
+  int32_t tile_n;                /* 0 = 256-wide tiles whenever N allows, 128 = narrow tiles                   */
+  int32_t pdl;                   /* 1: programmatic dependent launch along the kernel chain (process-wide)     */
+} marche_tuning;
+int marche_get_tuning(const marche_ctx* ctx, marche_tuning* out);
+/* MARCHE_EINVAL for a value outside the ranges above; nothing is enqueued. */
+int marche_set_tuning(marche_ctx* ctx, const marche_tuning* tuning);
 
 /* ---------------------------------------------------------------- diagnostics */
 const char* marche_strerror(int code);
@@ -435,6 +472,16 @@ const char* marche_last_error(const marche_ctx* ctx);
  * invalid).  It lives in pinned host memory owned by the context; synchronise
  * the stream before reading it. */
 int marche_device_status(const marche_ctx* ctx);
+/* Waits for `stream` and reports whether any kernel of this context gave up a bounded wait since the
+ * status word was last cleared: MARCHE_ETIMEOUT (the results of the calls enqueued since then are
+ * invalid; marche_device_status() names the kernel) or MARCHE_OK.  Synchronous.  The other
+ * synchronous calls, marche_validate_indices and marche_profile_end, report the same condition. */
+int marche_check_status(marche_ctx* ctx, marche_stream stream);
+/* Test hook for that path: enqueues a one-warp kernel whose single waiting thread uses the library's
+ * bounded wait on a barrier that nothing arrives on.  After `limit_cycles` SM clock cycles (1 ..
+ * 2e9; a million is about half a millisecond) the wait gives up, the status word is set and the
+ * kernel returns; nothing traps and the context stays usable.  Asynchronous. */
+int marche_debug_bounded_wait(marche_ctx* ctx, long long limit_cycles, marche_stream stream);
 /* Number of kernels this context has launched so far. */
 unsigned long long marche_launch_count(const marche_ctx* ctx);
 /* Per-kernel-class device time of the calls made between marche_profile_begin and

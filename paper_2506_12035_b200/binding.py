@@ -16,7 +16,9 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmarche.so")
 
-MARCHE_F32, MARCHE_BF16 = 0, 1
+MARCHE_F32, MARCHE_BF16, MARCHE_BF16_F16OP = 0, 1, 2
+ATTENTION_AUTO, ATTENTION_MMA, ATTENTION_TCGEN05 = 0, 1, 2
+GEMM_AUTO, GEMM_SINGLE, GEMM_PAIR = 0, 1, 2
 EPI_BIAS, EPI_BIAS_RESIDUAL, EPI_BIAS_GELU = 0, 1, 2
 ERRORS = {-1: "EINVAL", -2: "ESHAPE", -3: "EWORKSPACE", -4: "ECACHE", -5: "EINDEX", -6: "ECUDA", -7: "ETIMEOUT"}
 
@@ -40,6 +42,11 @@ MAR_FIELDS = ("enc_norm_g", "enc_norm_b", "w_dec_embed", "b_dec_embed", "mask_to
 
 class MarcheMarWeights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in MAR_FIELDS]
+
+
+class MarcheTuning(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("stream_k", "fuse_qkv_scatter", "attention_kernel", "attention_tc_min_rows",
+                                         "two_segment_attention", "gemm_kernel", "tail_split", "tile_n", "pdl")]
 
 
 class MarcheError(RuntimeError):
@@ -86,6 +93,10 @@ _SIGNATURES = {
     "marche_last_error": (C.c_char_p, [_vp]),
     "marche_device_status": (C.c_int, [_vp]),
     "marche_clear_device_status": (None, [_vp]),
+    "marche_get_tuning": (C.c_int, [_vp, C.POINTER(MarcheTuning)]),
+    "marche_set_tuning": (C.c_int, [_vp, C.POINTER(MarcheTuning)]),
+    "marche_check_status": (C.c_int, [_vp, _vp]),
+    "marche_debug_bounded_wait": (C.c_int, [_vp, C.c_longlong, _vp]),
 }
 EXPORTED_SYMBOLS = tuple(_SIGNATURES)
 
@@ -119,32 +130,51 @@ def _stream(stream: Optional[torch.cuda.Stream]) -> Optional[int]:
     return s.cuda_stream or None
 
 
-def upload_weights(blocks: Sequence[Dict], dtype: str, device="cuda") -> List[Dict[str, torch.Tensor]]:
-    """Copies per-block parameter arrays (NumPy or torch, fp32) to the device: the four
-    matrices as projection operands (fp16 in 16-bit mode, else fp32), LayerNorm parameters and
-    biases in fp32."""
-    mt = torch.float16 if dtype == "bf16" else torch.float32
+def _operand_dtype(dtype: str, operand: str) -> torch.dtype:
+    if dtype != "bf16":
+        return torch.float32
+    if operand not in ("f16", "bf16"):
+        raise ValueError("operand must be 'f16' or 'bf16'")
+    return torch.float16 if operand == "f16" else torch.bfloat16
+
+
+def _as_operand(t: torch.Tensor, mt: torch.dtype, name: str, device) -> torch.Tensor:
+    out = t.to(device=device, dtype=mt).contiguous()
+    if mt == torch.float16 and not bool(torch.isfinite(out).all()):
+        raise ValueError("%s does not fit IEEE fp16 (|value| > 65504); use operand='bf16'" % name)
+    return out
+
+
+def upload_weights(blocks: Sequence[Dict], dtype: str, device="cuda", operand: str = "f16") -> List[Dict[str, torch.Tensor]]:
+    """Copies per-block parameter arrays (NumPy or torch, fp32) to the device: the four matrices
+    in the projections' operand type (16-bit contexts: fp16 for operand "f16", bf16 for "bf16";
+    fp32 otherwise), LayerNorm parameters and biases in fp32."""
+    mt = _operand_dtype(dtype, operand)
     out = []
     for blk in blocks:
         d = {}
         for name in BLOCK_FIELDS:
             t = torch.as_tensor(blk[name])
-            d[name] = t.to(device=device, dtype=mt if name in MATRIX_FIELDS else torch.float32).contiguous()
+            d[name] = _as_operand(t, mt, name, device) if name in MATRIX_FIELDS else \
+                t.to(device=device, dtype=torch.float32).contiguous()
         out.append(d)
     return out
 
 
-def upload_mar_weights(mar: Dict, dtype: str, device="cuda") -> Dict[str, torch.Tensor]:
+def upload_mar_weights(mar: Dict, dtype: str, device="cuda", operand: str = "f16") -> Dict[str, torch.Tensor]:
     """Copies the two-stage model's glue parameters to the device (the encoder-to-decoder matrix
     as a projection operand, everything else fp32)."""
-    mt = torch.float16 if dtype == "bf16" else torch.float32
-    return {name: torch.as_tensor(mar[name]).to(device=device, dtype=mt if name == "w_dec_embed" else torch.float32)
-            .contiguous() for name in MAR_FIELDS}
+    mt = _operand_dtype(dtype, operand)
+    return {name: (_as_operand(torch.as_tensor(mar[name]), mt, name, device) if name == "w_dec_embed" else
+                   torch.as_tensor(mar[name]).to(device=device, dtype=torch.float32).contiguous())
+            for name in MAR_FIELDS}
 
 
 class Marche:
     """One model shape on the current CUDA device.  Methods carry the names of the C
-    calls without the `marche_` prefix and take torch CUDA tensors."""
+    calls without the `marche_` prefix and take torch CUDA tensors.  dtype "f32" or "bf16"; for
+    "bf16" the projections' operand type is taken from the weight matrices handed over (fp16 ->
+    MARCHE_BF16_F16OP, bf16 -> MARCHE_BF16)."""
 
     def __init__(self, *, L: int, E: int, D: int, H: int, F: int, S: int, B: int, dtype: str,
                  weights: Sequence[Dict[str, torch.Tensor]], n_buffer: int = 0, score_layer: int = -1,
@@ -155,11 +185,12 @@ class Marche:
         self.L, self.E, self.D, self.H, self.F, self.S, self.B = L, E, D, H, F, S, B
         self.dtype = dtype
         self.torch_dtype = torch.bfloat16 if dtype == "bf16" else torch.float32      # q/k/v, K/V cache
-        self.operand_dtype = torch.float16 if dtype == "bf16" else torch.float32     # projection operands
+        self.operand_dtype = weights[0]["w_qkv"].dtype if dtype == "bf16" else torch.float32   # projection operands
+        assert self.operand_dtype in ((torch.float16, torch.bfloat16) if dtype == "bf16" else (torch.float32,))
+        code = MARCHE_F32 if dtype != "bf16" else (MARCHE_BF16 if self.operand_dtype == torch.bfloat16 else MARCHE_BF16_F16OP)
         self.weights = list(weights)          # keeps the device tensors alive
         assert len(self.weights) == L
-        cfg = MarcheConfig(L, E, D, H, D // H, F, S, n_buffer, B, MARCHE_BF16 if dtype == "bf16" else MARCHE_F32,
-                           score_layer, ln_eps)
+        cfg = MarcheConfig(L, E, D, H, D // H, F, S, n_buffer, B, code, score_layer, ln_eps)
         arr = (MarcheBlockWeights * L)()
         for l, blk in enumerate(self.weights):
             for name in BLOCK_FIELDS:
@@ -186,7 +217,7 @@ class Marche:
     def _check(self, rc: int, h="self"):
         if rc != 0:
             detail = ""
-            if h == "self" and rc == -6:
+            if h == "self" and rc in (-1, -6):
                 detail = self.lib.marche_last_error(self.h).decode()
             raise MarcheError(rc, detail)
 
@@ -365,6 +396,28 @@ class Marche:
         cnt = (C.c_int * n)()
         self._check(self.lib.marche_profile_end(self.h, _stream(stream), ms, cnt))
         return {self.lib.marche_kernel_class_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n)}
+
+    def get_tuning(self) -> Dict[str, int]:
+        t = MarcheTuning()
+        self._check(self.lib.marche_get_tuning(self.h, C.byref(t)))
+        return {n: int(getattr(t, n)) for n, _ in MarcheTuning._fields_}
+
+    def set_tuning(self, **fields):
+        """Changes the named switches (see marche_tuning in the header); the others keep their values."""
+        t = MarcheTuning()
+        self._check(self.lib.marche_get_tuning(self.h, C.byref(t)))
+        for n, v in fields.items():
+            if n not in dict(MarcheTuning._fields_):
+                raise KeyError(n)
+            setattr(t, n, int(v))
+        self._check(self.lib.marche_set_tuning(self.h, C.byref(t)))
+
+    def check_status(self, stream=None):
+        """Synchronises and raises MarcheError(ETIMEOUT) if a kernel gave up a bounded wait."""
+        self._check(self.lib.marche_check_status(self.h, _stream(stream)))
+
+    def debug_bounded_wait(self, limit_cycles: int, stream=None):
+        self._check(self.lib.marche_debug_bounded_wait(self.h, limit_cycles, _stream(stream)))
 
     def device_status(self) -> int:
         return self.lib.marche_device_status(self.h)

@@ -12,7 +12,6 @@
 
 #include <cmath>
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -21,6 +20,7 @@
 
 #include "../../include/marche.h"
 #include "kernels.h"
+#include "launch_pdl.h"
 
 using namespace marche;
 
@@ -30,20 +30,14 @@ struct marche_ctx {
   marche_mar_weights mar{};                           // glue of the two-stage model (marche_set_mar_weights)
   bool has_mar = false;
   int device = 0;
-  bool bf16 = false;
+  bool bf16 = false;                                  // 16-bit context: q/k/v and the cache are bf16
+  bool a_bf16 = false;                                // ... and the projections' operands are bf16 too (else fp16)
+  int a_kind = OUT_F32;                               // element type of LayerNorm / attention / GELU outputs
   size_t eb = 4;
   float eps = 1e-6f;
   int score_layer = 0;
   std::vector<int> extra_score_layers;                // blocks that also accumulate scores (analysis only)
-  bool force_simt = false;
-  bool stream_k = true;                               // MARCHE_STREAM_K=0: whole tiles only in the residual GEMMs
-  bool fuse_qkv_scatter = true;                       // MARCHE_FUSE_QKV_SCATTER=0: separate scatter_kv launch
-  bool fuse_writeback = false;                        // MARCHE_FUSE_WB=1: write-back fused into the attention prologue
-                                                      // (measured slower: +11.7 us attention vs -10.5 us scatter_kv launch)
-  int attn_tc = -1;                                   // -1 auto, 0 never, 1 always (MARCHE_ATTN_TC)
-  int attn_tc_min_rows = 96;                          // auto: tcgen05 attention above this many active rows
-  int attn_mode = 0;                                  // 0 write-back kernel + one-segment attention, 1 two-segment (MARCHE_ATTN)
-  int gemm_mode = 0;                                  // 0 auto, 1 single-CTA MMA, 2 CTA-pair MMA (MARCHE_GEMM)
+  marche_tuning tune;                                 // kernel-selection switches (marche_set_tuning)
   std::vector<std::pair<const void*, bool>> caches;  // (cache pointer, filled)
   int* status_host = nullptr;                         // pinned, mapped
   int* status_dev = nullptr;
@@ -111,6 +105,55 @@ void mark(marche_ctx* ctx, int cls, cudaStream_t st) {
   ctx->event_class.push_back(cls);
 }
 
+marche_tuning default_tuning() {
+  marche_tuning t;
+  t.stream_k = 1;
+  t.fuse_qkv_scatter = 1;
+  t.attention_kernel = MARCHE_ATTENTION_AUTO;
+  t.attention_tc_min_rows = 96;
+  t.two_segment_attention = 0;
+  t.gemm_kernel = MARCHE_GEMM_AUTO;
+  t.tail_split = 1;
+  t.tile_n = 0;
+  t.pdl = 1;
+  return t;
+}
+
+// Every call that touches the device starts here: the context belongs to the device that was
+// current at marche_create, and its pointers mean nothing on another one.
+int enter(marche_ctx* ctx) {
+  if (!ctx) return MARCHE_EINVAL;
+  int dev = -1;
+  const cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaGetDevice");
+  if (dev != ctx->device) {
+    char msg[128];
+    snprintf(msg, sizeof msg, "the context was created on device %d but device %d is current", ctx->device, dev);
+    ctx->last_error = msg;
+    return MARCHE_EINVAL;
+  }
+  return MARCHE_OK;
+}
+#define MARCHE_ENTER(ctx)        \
+  do {                           \
+    const int rc__ = enter(ctx); \
+    if (rc__) return rc__;       \
+  } while (0)
+
+int misaligned(marche_ctx* ctx, const char* what) {
+  ctx->last_error = std::string(what) + ": a 16-bit context needs 16-byte aligned operands and row strides "
+                    "that are multiples of 8 elements (there is no slow path to fall back to)";
+  return MARCHE_EINVAL;
+}
+
+GemmTuning gemm_tuning(const marche_ctx* ctx) {
+  GemmTuning g;
+  g.stream_k = ctx->tune.stream_k != 0;
+  g.tail_split = ctx->tune.tail_split;
+  g.tile_n = ctx->tune.tile_n;
+  return g;
+}
+
 int refresh_count(float ratio, int S, int n_cand) {
   const int want = (int)std::floor((double)ratio * (double)S + 0.5);
   return want < n_cand ? (want < 0 ? 0 : want) : n_cand;
@@ -129,24 +172,29 @@ int score_slot(const marche_ctx* ctx, int l) {
 // whole 256-column tiles per q / K / V range, 32-bit cache offsets): no scatter_kv launch then.
 bool qkv_scatter_fused(const marche_ctx* ctx, int M, int S) {
   const marche_config& c = ctx->cfg;
-  return ctx->fuse_qkv_scatter && ctx->bf16 && !ctx->force_simt && ctx->attn_mode == 0 && !ctx->fuse_writeback &&
-         (ctx->gemm_mode == 2 || (ctx->gemm_mode == 0 && M > 128)) && c.width % 256 == 0 &&
+  return ctx->tune.fuse_qkv_scatter && ctx->bf16 && !ctx->tune.two_segment_attention && ctx->tune.tile_n != 128 &&
+         (ctx->tune.gemm_kernel == MARCHE_GEMM_PAIR || (ctx->tune.gemm_kernel == MARCHE_GEMM_AUTO && M > 128)) &&
+         c.width % 256 == 0 &&
          (long)2 * c.batch * S * c.width < (1L << 31);
 }
 
 int do_linear(marche_ctx* ctx, int cls, const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
               int epi, void* out, cudaStream_t st, int* turn = nullptr, const KvScatter* kv = nullptr) {
+  if (!ctx->bf16) {
+    if (M > 0) mark(ctx, cls, st);
+    MARCHE_TRY(launch_gemm_simt((const float*)a, lda, M, (const float*)w, bias, N, K, epi, (float*)out, st), "gemm");
+    return MARCHE_OK;
+  }
+  // 16-bit contexts run on the tensor cores or not at all
+  if (N % 128 || K % 64) return MARCHE_ESHAPE;
+  if (lda % 8 || (((uintptr_t)a | (uintptr_t)w | (uintptr_t)out) & 15)) return misaligned(ctx, "projection");
   if (M > 0) mark(ctx, cls, st);
-  const bool tc = ctx->bf16 && !ctx->force_simt && N % 128 == 0 && K % 64 == 0 && lda % 8 == 0 &&
-                  (((uintptr_t)a | (uintptr_t)w | (uintptr_t)out) & 15) == 0;
-  const bool pair = tc && (ctx->gemm_mode == 2 || (ctx->gemm_mode == 0 && M > 128));
+  const bool pair = ctx->tune.gemm_kernel == MARCHE_GEMM_PAIR || (ctx->tune.gemm_kernel == MARCHE_GEMM_AUTO && M > 128);
   if (pair)
-    MARCHE_TRY(launch_gemm_tcgen05_2cta(a, lda, M, w, bias, N, K, epi, out, ctx->status_dev, st,
-                                        ctx->stream_k ? turn : nullptr, kv), "gemm_tcgen05_2cta");
-  else if (tc)
-    MARCHE_TRY(launch_gemm_tcgen05(a, lda, M, w, bias, N, K, epi, out, ctx->status_dev, st), "gemm_tcgen05");
+    MARCHE_TRY(launch_gemm_tcgen05_2cta(a, lda, M, w, bias, N, K, epi, out, ctx->a_bf16, ctx->status_dev, st,
+                                        gemm_tuning(ctx), turn, kv), "gemm_tcgen05_2cta");
   else
-    MARCHE_TRY(launch_gemm_simt(ctx->bf16, a, lda, M, w, bias, N, K, epi, out, st), "gemm");
+    MARCHE_TRY(launch_gemm_tcgen05(a, lda, M, w, bias, N, K, epi, out, ctx->a_bf16, ctx->status_dev, st), "gemm_tcgen05");
   return MARCHE_OK;
 }
 
@@ -154,26 +202,29 @@ int do_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void* ca
                  float* partial, void* o, cudaStream_t st, int S_kv = 0) {
   const marche_config& c = ctx->cfg;
   const int S = S_kv > 0 ? S_kv : c.seq_len;            // tokens per sample in cache_layer [2][B][S][D]
+  if (!ctx->bf16) {
+    if (n > 0) mark(ctx, MARCHE_KC_ATTENTION, st);
+    MARCHE_TRY(launch_attention_simt((const float*)q, ld_q, c.batch, n, S, c.n_heads, c.head_dim, (const float*)cache_layer,
+                                     is_new, partial, (float*)o, st), "attention");
+    return MARCHE_OK;
+  }
+  if (ld_q % 2 || ((uintptr_t)q & 3) || ((uintptr_t)cache_layer & 15) || ((uintptr_t)o & 15)) return misaligned(ctx, "attention");
   if (n > 0) mark(ctx, MARCHE_KC_ATTENTION, st);
-  const bool tc = ctx->bf16 && !ctx->force_simt && (c.head_dim == 64 || c.head_dim == 80) && ld_q % 2 == 0 &&
-                  ((uintptr_t)q & 3) == 0 && ((uintptr_t)cache_layer & 15) == 0;
   // Two tensor-core kernels.  At small active sets the step is bound by streaming the cache and the
   // mma.sync kernel (several small CTAs per SM, one pass) is faster: 41 us vs 69 us at n = 41.  Once
   // the legacy tensor path saturates (about 250 TFLOP/s) the tcgen05 kernel wins: 109 vs 172 us at
   // n = 122 (S 1088), 840 vs 1100 us at n = S = 1088, and earlier for the two-pass scoring flavour
-  // (97 vs 143 us at n = 77).  MARCHE_ATTN_TC=0 / 1 forces one of them; head_dim 80 has only the former.
-  const int tc_min = is_new ? 64 : ctx->attn_tc_min_rows;
-  const bool tc5 = tc && c.head_dim == 64 && ld_q % 8 == 0 && ((uintptr_t)q & 15) == 0 &&
-                   (ctx->attn_tc == 1 || (ctx->attn_tc < 0 && n > tc_min));
+  // (97 vs 143 us at n = 77).  marche_tuning.attention_kernel forces one of them; head_dim 80 has only the former.
+  const int tc_min = is_new ? 64 : ctx->tune.attention_tc_min_rows;
+  const bool tc5 = c.head_dim == 64 && ld_q % 8 == 0 && ((uintptr_t)q & 15) == 0 &&
+                   (ctx->tune.attention_kernel == MARCHE_ATTENTION_TCGEN05 ||
+                    (ctx->tune.attention_kernel == MARCHE_ATTENTION_AUTO && n > tc_min));
   if (tc5)
     MARCHE_TRY(launch_attention_tcgen05(q, ld_q, c.batch, n, S, c.n_heads, c.head_dim, cache_layer, is_new,
-                                        partial, o, ctx->status_dev, st), "attention_tcgen05");
-  else if (tc)
-    MARCHE_TRY(launch_attention_mma(q, ld_q, c.batch, n, S, c.n_heads, c.head_dim, cache_layer, is_new,
-                                    partial, o, ctx->status_dev, st), "attention_mma");
+                                        partial, o, ctx->a_bf16, ctx->status_dev, st), "attention_tcgen05");
   else
-    MARCHE_TRY(launch_attention_simt(ctx->bf16, q, ld_q, c.batch, n, S, c.n_heads, c.head_dim, cache_layer,
-                                     is_new, partial, o, st), "attention");
+    MARCHE_TRY(launch_attention_mma(q, ld_q, c.batch, n, S, c.n_heads, c.head_dim, cache_layer, is_new,
+                                    partial, o, ctx->a_bf16, ctx->status_dev, st), "attention_mma");
   return MARCHE_OK;
 }
 
@@ -224,10 +275,10 @@ int run_blocks(marche_ctx* ctx, int l_begin, int l_end, const float* gather_src,
     float* partial_l = bf.partial + (size_t)(slot > 0 ? slot : 0) * B * c.n_heads * c.seq_len;
     mark(ctx, MARCHE_KC_GATHER_LN, st);
     if (l == l_begin && gather_src)
-      MARCHE_TRY(launch_gather_layernorm(ctx->bf16, gather_src, src_rows, idx, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
+      MARCHE_TRY(launch_gather_layernorm(ctx->a_kind, gather_src, src_rows, idx, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
                                          x, bf.u, st), "gather_layernorm");
     else
-      MARCHE_TRY(launch_gather_layernorm(ctx->bf16, x, nA, nullptr, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
+      MARCHE_TRY(launch_gather_layernorm(ctx->a_kind, x, nA, nullptr, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
                                          nullptr, bf.u, st), "layernorm1");
     const bool fused_kv = qkv_scatter_fused(ctx, M, S);
     const KvScatter kvs = {kv_idx, cache_l, nA, S, B, D};
@@ -238,20 +289,12 @@ int run_blocks(marche_ctx* ctx, int l_begin, int l_end, const float* gather_src,
       // the projection's epilogue has written K and V into the cache (Algorithm 1 line 11)
       rc = do_attention(ctx, bf.qkv, 3 * D, nA, cache_l, flags_l, partial_l, bf.o, st, S);
       if (rc) return rc;
-    } else if (ctx->attn_mode == 1 && ctx->bf16 && !ctx->force_simt) {
+    } else if (ctx->tune.two_segment_attention && ctx->bf16) {
       // two-segment attention: fresh K/V read in place, cache write-back by the same kernel
       mark(ctx, MARCHE_KC_ATTENTION, st);
       MARCHE_TRY(launch_attention_twoseg(bf.qkv, 3 * D, D, 2 * D, B, nA, S, c.n_heads, c.head_dim, kv_idx, cache_l,
-                                         flags_l, partial_l, bf.o, ctx->status_dev, st),
+                                         flags_l, partial_l, bf.o, ctx->a_bf16, ctx->status_dev, st),
                  "attention_twoseg");
-    } else if (ctx->fuse_writeback && ctx->bf16 && !ctx->force_simt && ctx->attn_tc != 1 &&
-               !(c.head_dim == 64 && ctx->attn_tc < 0 &&
-                 nA > (flags_l ? 64 : ctx->attn_tc_min_rows))) {
-      // mma.sync attention with the cache write-back fused into its prologue (no scatter_kv launch)
-      mark(ctx, MARCHE_KC_ATTENTION, st);
-      MARCHE_TRY(launch_attention_mma(bf.qkv, 3 * D, B, nA, S, c.n_heads, c.head_dim, cache_l,
-                                      flags_l, partial_l, bf.o, ctx->status_dev, st,
-                                      true, kv_idx, D, 2 * D), "attention_mma_wb");
     } else {
       mark(ctx, MARCHE_KC_SCATTER_KV, st);
       MARCHE_TRY(launch_scatter_kv(ctx->bf16, bf.qkv + (size_t)D * eb, bf.qkv + (size_t)2 * D * eb, 3 * D, kv_idx, B, nA,
@@ -263,7 +306,7 @@ int run_blocks(marche_ctx* ctx, int l_begin, int l_end, const float* gather_src,
     rc = do_linear(ctx, MARCHE_KC_GEMM_O, bf.o, D, M, bw.w_o, bw.b_o, D, D, MARCHE_EPI_BIAS_RESIDUAL, x, st, bf.turn);
     if (rc) return rc;
     mark(ctx, MARCHE_KC_GATHER_LN, st);
-    MARCHE_TRY(launch_gather_layernorm(ctx->bf16, x, nA, nullptr, B, nA, D, bw.ln2_g, bw.ln2_b, ctx->eps, nullptr,
+    MARCHE_TRY(launch_gather_layernorm(ctx->a_kind, x, nA, nullptr, B, nA, D, bw.ln2_g, bw.ln2_b, ctx->eps, nullptr,
                                        bf.u, st), "layernorm2");
     rc = do_linear(ctx, MARCHE_KC_GEMM_FC1, bf.u, D, M, bw.w_fc1, bw.b_fc1, F, D, MARCHE_EPI_BIAS_GELU, bf.g, st);
     if (rc) return rc;
@@ -281,6 +324,7 @@ int run_stack(marche_ctx* ctx, const float* hidden, void* kv_cache, const int32_
   const marche_config& c = ctx->cfg;
   const int B = c.batch, S = c.seq_len, D = c.width, H = c.n_heads, L = c.n_blocks;
   if (!hidden || !kv_cache || !hidden_out || !workspace || hidden == hidden_out) return MARCHE_EINVAL;
+  if (((uintptr_t)hidden | (uintptr_t)hidden_out | (uintptr_t)kv_cache) & 15) return MARCHE_EINVAL;
   if (nA < 1 || nA > S || n_new < 0 || n_new > nA || n_excl < 0 || n_new + n_excl > S) return MARCHE_EINVAL;
   if ((n_new > 0 && !new_idx) || (n_excl > 0 && !excl_idx)) return MARCHE_EINVAL;
   if (((uintptr_t)workspace & 255) != 0) return MARCHE_EINVAL;
@@ -291,7 +335,7 @@ int run_stack(marche_ctx* ctx, const float* hidden, void* kv_cache, const int32_
   const StackBufs bf = carve(workspace, w);
 
   // the workspace is scratch between calls: make sure the stream-K turn flags start at zero
-  if (ctx->bf16 && ctx->stream_k) MARCHE_TRY(cudaMemsetAsync(bf.turn, 0, w.turn_bytes, st), "memset");
+  if (ctx->bf16 && ctx->tune.stream_k) MARCHE_TRY(cudaMemsetAsync(bf.turn, 0, w.turn_bytes, st), "memset");
   mark(ctx, MARCHE_KC_FLAGS, st);
   MARCHE_TRY(launch_step_flags(active_idx, nA, new_idx, n_new, excl_idx, n_excl, B, S, bf.is_new, bf.cand, st), "flags");
   const int rc = run_blocks(ctx, 0, L, hidden, S, active_idx, nA, bf.x, bf, kv_cache, bf.is_new, st);
@@ -312,6 +356,7 @@ int run_in_step(marche_ctx* ctx, const float* hidden, void* kv_cache, const int3
   const int B = c.batch, S = c.seq_len, D = c.width, H = c.n_heads, L = c.n_blocks, sl = ctx->score_layer;
   if (!hidden || !kv_cache || !hidden_out || !workspace || !refresh_idx || !active_idx || hidden == hidden_out)
     return MARCHE_EINVAL;
+  if (((uintptr_t)hidden | (uintptr_t)hidden_out | (uintptr_t)kv_cache) & 15) return MARCHE_EINVAL;
   if (n_new < 0 || n_prev < 0 || k < 0 || n_new + n_prev + k > S || n_new + n_prev + k < 1) return MARCHE_EINVAL;
   if ((n_new > 0 && !new_idx) || (n_prev > 0 && !prev_idx)) return MARCHE_EINVAL;
   if (sl >= L - 1) return MARCHE_EINVAL;                     // needs at least one cache-aware block
@@ -320,7 +365,7 @@ int run_in_step(marche_ctx* ctx, const float* hidden, void* kv_cache, const int3
   if (ws_bytes < w.total) return MARCHE_EWORKSPACE;
   const StackBufs bf = carve(workspace, w);
   const int nA = n_new + n_prev + k;
-  if (ctx->bf16 && ctx->stream_k) MARCHE_TRY(cudaMemsetAsync(bf.turn, 0, w.turn_bytes, st), "memset");
+  if (ctx->bf16 && ctx->tune.stream_k) MARCHE_TRY(cudaMemsetAsync(bf.turn, 0, w.turn_bytes, st), "memset");
 
   // phase 1: every token; generating rows flagged for the scores; candidates = all \ (new u prev)
   mark(ctx, MARCHE_KC_FLAGS, st);
@@ -352,6 +397,7 @@ int run_mar(marche_ctx* ctx, bool full_decoder, const float* tokens, const int32
   const int sl = ctx->score_layer;
   if (!ctx->has_mar) return MARCHE_EINVAL;
   if (!tokens || !known_idx || !kv_cache || !z_out || !workspace || tokens == z_out) return MARCHE_EINVAL;
+  if (((uintptr_t)tokens | (uintptr_t)z_out | (uintptr_t)kv_cache) & 15) return MARCHE_EINVAL;
   if (E < 1 || E >= L || sl < E) return MARCHE_EINVAL;
   if (n_known < 1 || n_known > S || n_new < 0 || n_prev < 0 || k < 0 || n_new + n_prev + k > S) return MARCHE_EINVAL;
   if ((n_new > 0 && !new_idx) || (n_prev > 0 && !prev_idx) || (k > 0 && !refresh_idx)) return MARCHE_EINVAL;
@@ -362,7 +408,7 @@ int run_mar(marche_ctx* ctx, bool full_decoder, const float* tokens, const int32
   if (ws_bytes < w.total) return MARCHE_EWORKSPACE;
   const StackBufs bf = carve(workspace, w);
   const marche_mar_weights& mw = ctx->mar;
-  if (ctx->bf16 && ctx->stream_k) MARCHE_TRY(cudaMemsetAsync(bf.turn, 0, w.turn_bytes, st), "memset");
+  if (ctx->bf16 && ctx->tune.stream_k) MARCHE_TRY(cudaMemsetAsync(bf.turn, 0, w.turn_bytes, st), "memset");
 
   mark(ctx, MARCHE_KC_FLAGS, st);
   MARCHE_TRY(launch_step_flags(nullptr, S, new_idx, n_new, prev_idx, n_prev, B, S, bf.is_new, bf.cand, st), "flags");
@@ -371,7 +417,7 @@ int run_mar(marche_ctx* ctx, bool full_decoder, const float* tokens, const int32
   if (rc) return rc;
   // ---- Eq. 2: x3[b][s] = mask + pos[s];  x3[b][known] = W_de * LN(h_enc) + b_de + pos[known]
   mark(ctx, MARCHE_KC_GATHER_LN, st);
-  MARCHE_TRY(launch_gather_layernorm(ctx->bf16, bf.x, n_known, nullptr, B, n_known, D, mw.enc_norm_g, mw.enc_norm_b,
+  MARCHE_TRY(launch_gather_layernorm(ctx->a_kind, bf.x, n_known, nullptr, B, n_known, D, mw.enc_norm_g, mw.enc_norm_b,
                                      ctx->eps, nullptr, bf.u, st), "encoder_norm");
   mark(ctx, MARCHE_KC_OTHER, st);
   MARCHE_TRY(launch_gather_table_rows(mw.dec_pos, known_idx, (long)B * n_known, D, bf.x2, st), "gather_table_rows");
@@ -390,7 +436,7 @@ int run_mar(marche_ctx* ctx, bool full_decoder, const float* tokens, const int32
     mark(ctx, MARCHE_KC_TOPK, st);
     MARCHE_TRY(launch_topk(bf.partial, H, bf.scores, bf.cand, B, S, k, refresh_idx, st), "topk");
     mark(ctx, MARCHE_KC_GATHER_LN, st);
-    MARCHE_TRY(launch_gather_layernorm(false, bf.x, S, nullptr, B, S, D, mw.dec_norm_g, mw.dec_norm_b, ctx->eps,
+    MARCHE_TRY(launch_gather_layernorm(OUT_F32, bf.x, S, nullptr, B, S, D, mw.dec_norm_g, mw.dec_norm_b, ctx->eps,
                                        nullptr, z_out, st), "decoder_norm");
     return MARCHE_OK;
   }
@@ -404,7 +450,7 @@ int run_mar(marche_ctx* ctx, bool full_decoder, const float* tokens, const int32
   rc = run_blocks(ctx, sl + 1, L, bf.x, S, active_idx, nA, bf.x2, bf, kv_cache, nullptr, st);
   if (rc) return rc;
   mark(ctx, MARCHE_KC_GATHER_LN, st);
-  MARCHE_TRY(launch_gather_layernorm(false, bf.x2, nA, nullptr, B, nA, D, mw.dec_norm_g, mw.dec_norm_b, ctx->eps,
+  MARCHE_TRY(launch_gather_layernorm(OUT_F32, bf.x2, nA, nullptr, B, nA, D, mw.dec_norm_g, mw.dec_norm_b, ctx->eps,
                                      nullptr, z_out, st, active_idx, S), "decoder_norm");
   return MARCHE_OK;
 }
@@ -424,39 +470,32 @@ int marche_create(const marche_config* cfg, const marche_block_weights* blocks, 
   *out = nullptr;
   const marche_config& c = *cfg;
   if (c.n_blocks < 1 || c.batch < 1 || c.seq_len < 1 || c.n_heads < 1 || c.head_dim < 1) return MARCHE_EINVAL;
-  if (c.dtype != MARCHE_F32 && c.dtype != MARCHE_BF16) return MARCHE_EINVAL;
+  if (c.dtype != MARCHE_F32 && c.dtype != MARCHE_BF16 && c.dtype != MARCHE_BF16_F16OP) return MARCHE_EINVAL;
   if (c.width != c.n_heads * c.head_dim) return MARCHE_EINVAL;
   if (c.width % 128 || c.width > 2048 || c.mlp_dim % 128 || c.mlp_dim < 128 || c.seq_len > 2048)
     return MARCHE_ESHAPE;
   if (c.head_dim % 16 || c.head_dim > 128) return MARCHE_ESHAPE;
-  if (c.dtype == MARCHE_BF16 && c.head_dim != 64 && c.head_dim != 80) return MARCHE_ESHAPE;
+  if (c.dtype != MARCHE_F32 && c.head_dim != 64 && c.head_dim != 80) return MARCHE_ESHAPE;
   if (c.score_layer >= c.n_blocks) return MARCHE_EINVAL;
   marche_ctx* ctx = new (std::nothrow) marche_ctx();
   if (!ctx) return MARCHE_EINVAL;
   ctx->cfg = c;
   ctx->blocks.assign(blocks, blocks + c.n_blocks);
-  ctx->bf16 = c.dtype == MARCHE_BF16;
+  for (const marche_block_weights& b : ctx->blocks) {
+    // vector loads / TMA: every parameter array starts on a 16-byte boundary
+    const void* ptrs[12] = {b.ln1_g, b.ln1_b, b.w_qkv, b.b_qkv, b.w_o, b.b_o, b.ln2_g, b.ln2_b, b.w_fc1, b.b_fc1, b.w_fc2, b.b_fc2};
+    for (const void* q : ptrs)
+      if (!q || ((uintptr_t)q & 15)) { delete ctx; return MARCHE_EINVAL; }
+  }
+  ctx->bf16 = c.dtype != MARCHE_F32;
+  ctx->a_bf16 = c.dtype == MARCHE_BF16;
+  ctx->a_kind = !ctx->bf16 ? OUT_F32 : (ctx->a_bf16 ? OUT_BF16 : OUT_F16);
   ctx->eb = ctx->bf16 ? 2 : 4;
+  ctx->tune = default_tuning();
   ctx->eps = c.ln_eps > 0.f ? c.ln_eps : 1e-6f;
   int sl = c.score_layer >= 0 ? c.score_layer : c.n_enc_blocks + 1;
   if (sl >= c.n_blocks) sl = c.n_blocks - 1;
   ctx->score_layer = sl;
-  const char* fs = getenv("MARCHE_FORCE_SIMT");
-  ctx->force_simt = fs && fs[0] == '1';
-  const char* sk = getenv("MARCHE_STREAM_K");
-  ctx->stream_k = !(sk && sk[0] == '0');
-  const char* fq = getenv("MARCHE_FUSE_QKV_SCATTER");
-  ctx->fuse_qkv_scatter = !(fq && fq[0] == '0');
-  const char* fw = getenv("MARCHE_FUSE_WB");
-  ctx->fuse_writeback = fw && fw[0] == '1';
-  const char* tcv = getenv("MARCHE_ATTN_TC");
-  if (tcv) ctx->attn_tc = atoi(tcv);
-  const char* tcm = getenv("MARCHE_ATTN_TC_MIN");
-  if (tcm) ctx->attn_tc_min_rows = atoi(tcm);
-  const char* am = getenv("MARCHE_ATTN");
-  ctx->attn_mode = (am && (am[0] == '1' || am[0] == 't')) ? 1 : 0;
-  const char* gm = getenv("MARCHE_GEMM");
-  ctx->gemm_mode = gm ? atoi(gm) : 0;
   cudaError_t e = cudaGetDevice(&ctx->device);
   if (e == cudaSuccess) e = cudaHostAlloc((void**)&ctx->status_host, 64, cudaHostAllocMapped);
   if (e == cudaSuccess) {
@@ -492,6 +531,7 @@ size_t marche_workspace_bytes(const marche_ctx* ctx, int max_active) {
 
 int marche_init_cache(marche_ctx* ctx, void* kv_cache, size_t bytes, marche_stream stream) {
   if (!ctx || !kv_cache) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   if (bytes < marche_cache_bytes(ctx)) return MARCHE_EWORKSPACE;
   MARCHE_TRY(cudaMemsetAsync(kv_cache, 0, marche_cache_bytes(ctx), (cudaStream_t)stream), "memset");
   if (auto* e = find_cache(ctx, kv_cache)) e->second = false;
@@ -504,6 +544,7 @@ int marche_step(marche_ctx* ctx, const float* hidden, void* kv_cache, const int3
                 float* hidden_out, int32_t* refresh_idx, int* n_refresh, void* workspace, size_t workspace_bytes,
                 marche_stream stream) {
   if (!ctx || !active_idx) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   auto* e = find_cache(ctx, kv_cache);
   if (!e || !e->second) return MARCHE_ECACHE;
   return run_stack(ctx, hidden, kv_cache, active_idx, n_active, new_idx, n_new, exclude_idx, n_excl, refresh_ratio,
@@ -514,7 +555,7 @@ int marche_full_step(marche_ctx* ctx, const float* hidden, void* kv_cache, const
                      const int32_t* exclude_idx, int n_excl, float refresh_ratio, float* hidden_out,
                      int32_t* refresh_idx, int* n_refresh, void* workspace, size_t workspace_bytes,
                      marche_stream stream) {
-  if (!ctx) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   const int rc = run_stack(ctx, hidden, kv_cache, nullptr, ctx->cfg.seq_len, new_idx, n_new, exclude_idx, n_excl,
                            refresh_ratio, hidden_out, refresh_idx, n_refresh, workspace, workspace_bytes,
                            (cudaStream_t)stream);
@@ -529,7 +570,7 @@ int marche_step_in_step_selection(marche_ctx* ctx, const float* hidden, void* kv
                                   int n_new, const int32_t* prev_idx, int n_prev, int n_refresh,
                                   const int32_t* forced_refresh, float* hidden_out, int32_t* refresh_idx,
                                   int32_t* active_idx, void* workspace, size_t workspace_bytes, marche_stream stream) {
-  if (!ctx) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   auto* e = find_cache(ctx, kv_cache);
   if (!e || !e->second) return MARCHE_ECACHE;
   return run_in_step(ctx, hidden, kv_cache, new_idx, n_new, prev_idx, n_prev, n_refresh, forced_refresh, hidden_out,
@@ -541,6 +582,9 @@ int marche_set_mar_weights(marche_ctx* ctx, const marche_mar_weights* w) {
   if (!w->enc_norm_g || !w->enc_norm_b || !w->w_dec_embed || !w->b_dec_embed || !w->mask_token || !w->dec_pos ||
       !w->dec_norm_g || !w->dec_norm_b)
     return MARCHE_EINVAL;
+  if (((uintptr_t)w->enc_norm_g | (uintptr_t)w->enc_norm_b | (uintptr_t)w->w_dec_embed | (uintptr_t)w->b_dec_embed |
+       (uintptr_t)w->mask_token | (uintptr_t)w->dec_pos | (uintptr_t)w->dec_norm_g | (uintptr_t)w->dec_norm_b) & 15)
+    return MARCHE_EINVAL;
   if (ctx->cfg.n_enc_blocks < 1 || ctx->cfg.n_enc_blocks >= ctx->cfg.n_blocks) return MARCHE_EINVAL;
   ctx->mar = *w;
   ctx->has_mar = true;
@@ -551,7 +595,7 @@ int marche_mar_step(marche_ctx* ctx, int full_decoder, const float* tokens, cons
                     void* kv_cache, const int32_t* new_idx, int n_new, const int32_t* prev_idx, int n_prev,
                     int n_refresh, const int32_t* forced_refresh, float* z_out, int32_t* refresh_idx,
                     int32_t* active_idx, void* workspace, size_t workspace_bytes, marche_stream stream) {
-  if (!ctx) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   auto* e = find_cache(ctx, kv_cache);
   if (!full_decoder && (!e || !e->second)) return MARCHE_ECACHE;
   const int rc = run_mar(ctx, full_decoder != 0, tokens, known_idx, n_known, kv_cache, new_idx, n_new, prev_idx, n_prev,
@@ -575,6 +619,7 @@ int marche_select_refresh_policy(marche_ctx* ctx, const float* scores, const int
                                  const int32_t* exclude_idx, int n_excl, int k, int policy, uint32_t seed,
                                  int32_t* refresh_idx, void* mask_scratch, marche_stream stream) {
   if (!ctx || !scores || !mask_scratch || n_new < 0 || n_excl < 0 || k < 0) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   if (policy < MARCHE_SELECT_HIGH || policy > MARCHE_SELECT_RANDOM) return MARCHE_EINVAL;
   if ((n_new > 0 && !new_idx) || (n_excl > 0 && !exclude_idx)) return MARCHE_EINVAL;
   const int B = ctx->cfg.batch, S = ctx->cfg.seq_len;
@@ -606,6 +651,7 @@ int marche_set_score_layers(marche_ctx* ctx, const int32_t* layers, int n) {
 
 int marche_get_layer_scores(marche_ctx* ctx, void* workspace, int layer, float* scores_out, marche_stream stream) {
   if (!ctx || !workspace || !scores_out) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   const int slot = score_slot(ctx, layer);
   if (slot < 0) return MARCHE_EINVAL;
   const marche_config& c = ctx->cfg;
@@ -620,6 +666,7 @@ int marche_get_layer_scores(marche_ctx* ctx, void* workspace, int layer, float* 
 
 int marche_get_scores(marche_ctx* ctx, const void* workspace, float* scores_out, marche_stream stream) {
   if (!ctx || !workspace || !scores_out) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   const size_t bytes = (size_t)ctx->cfg.batch * ctx->cfg.seq_len * sizeof(float);
   MARCHE_TRY(cudaMemcpyAsync(scores_out, (const char*)workspace + ws_layout(ctx, 1).scores, bytes,
                              cudaMemcpyDeviceToDevice, (cudaStream_t)stream), "memcpy");
@@ -629,6 +676,7 @@ int marche_get_scores(marche_ctx* ctx, const void* workspace, float* scores_out,
 int marche_build_active(marche_ctx* ctx, const int32_t* new_idx, int n_new, const int32_t* prev_idx, int n_prev,
                         const int32_t* refresh_idx, int n_refresh, int32_t* active_idx, marche_stream stream) {
   if (!ctx || !active_idx || n_new < 0 || n_prev < 0 || n_refresh < 0) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   if ((n_new && !new_idx) || (n_prev && !prev_idx) || (n_refresh && !refresh_idx)) return MARCHE_EINVAL;
   if (n_new + n_prev + n_refresh > ctx->cfg.seq_len) return MARCHE_EINVAL;
   mark(ctx, MARCHE_KC_OTHER, (cudaStream_t)stream);
@@ -640,6 +688,7 @@ int marche_build_active(marche_ctx* ctx, const int32_t* new_idx, int n_new, cons
 int marche_scatter_rows(marche_ctx* ctx, const float* rows, const int32_t* idx, int n, float* dst,
                         marche_stream stream) {
   if (!ctx || !rows || !dst || n < 0 || n > ctx->cfg.seq_len || (n && !idx)) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   if (n == 0) return MARCHE_OK;
   mark(ctx, MARCHE_KC_SCATTER_ROWS, (cudaStream_t)stream);
   MARCHE_TRY(launch_scatter_rows(rows, idx, ctx->cfg.batch, n, ctx->cfg.seq_len, ctx->cfg.width, dst,
@@ -650,6 +699,7 @@ int marche_scatter_rows(marche_ctx* ctx, const float* rows, const int32_t* idx, 
 int marche_validate_indices(marche_ctx* ctx, const int32_t* active_idx, int n_active, const int32_t* new_idx,
                             int n_new, const int32_t* exclude_idx, int n_excl, marche_stream stream) {
   if (!ctx || n_active < 0 || n_new < 0 || n_excl < 0) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   if ((n_active && !active_idx) || (n_new && !new_idx) || (n_excl && !exclude_idx)) return MARCHE_EINVAL;
   const int S = ctx->cfg.seq_len;
   if (n_active > S || n_new > S || n_excl > S) return MARCHE_EINDEX;
@@ -659,6 +709,7 @@ int marche_validate_indices(marche_ctx* ctx, const int32_t* active_idx, int n_ac
   MARCHE_TRY(launch_validate(n_active ? active_idx : nullptr, n_active, new_idx, n_new, exclude_idx, n_excl,
                              ctx->cfg.batch, S, ctx->status_dev + 8, st), "validate");
   MARCHE_TRY(cudaStreamSynchronize(st), "sync");
+  if (*(volatile int*)ctx->status_host) return MARCHE_ETIMEOUT;   // an earlier kernel of the stream gave up a wait
   return *flag ? MARCHE_EINDEX : MARCHE_OK;
 }
 
@@ -666,9 +717,10 @@ int marche_gather_layernorm(marche_ctx* ctx, const float* src, int src_rows, con
                             const float* gamma, const float* beta, float* x_out, void* u_out,
                             marche_stream stream) {
   if (!ctx || !src || !gamma || !beta || !u_out || n < 0 || src_rows < 1) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   if (!idx && n > src_rows) return MARCHE_EINVAL;
   mark(ctx, MARCHE_KC_GATHER_LN, (cudaStream_t)stream);
-  MARCHE_TRY(launch_gather_layernorm(ctx->bf16, src, src_rows, idx, ctx->cfg.batch, n, ctx->cfg.width, gamma, beta,
+  MARCHE_TRY(launch_gather_layernorm(ctx->a_kind, src, src_rows, idx, ctx->cfg.batch, n, ctx->cfg.width, gamma, beta,
                                      ctx->eps, x_out, u_out, (cudaStream_t)stream), "gather_layernorm");
   return MARCHE_OK;
 }
@@ -677,6 +729,7 @@ int marche_linear(marche_ctx* ctx, const void* a, int lda, int M, const void* w,
                   int epilogue, void* out, marche_stream stream) {
   if (!ctx || !a || !w || !bias || !out || M < 0 || N < 1 || K < 1 || lda < K) return MARCHE_EINVAL;
   if (epilogue < 0 || epilogue > 2) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   if (ctx->bf16 ? (N % 128 || K % 64 || lda % 8) : (N % 64 || K % 16 || lda % 4)) return MARCHE_ESHAPE;
   return do_linear(ctx, MARCHE_KC_OTHER, a, lda, M, w, bias, N, K, epilogue, out, (cudaStream_t)stream);
 }
@@ -686,6 +739,7 @@ int marche_scatter_kv(marche_ctx* ctx, const void* k, const void* v, int ld_kv, 
   if (!ctx || !k || !v || !cache_layer || n < 0 || n > ctx->cfg.seq_len || ld_kv < ctx->cfg.width)
     return MARCHE_EINVAL;
   if (!idx && n != ctx->cfg.seq_len) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   mark(ctx, MARCHE_KC_SCATTER_KV, (cudaStream_t)stream);
   MARCHE_TRY(launch_scatter_kv(ctx->bf16, k, v, ld_kv, idx, ctx->cfg.batch, n, ctx->cfg.seq_len, ctx->cfg.width,
                                cache_layer, (cudaStream_t)stream), "scatter_kv");
@@ -700,11 +754,12 @@ int marche_attention_two_segment(marche_ctx* ctx, const void* qkv, int ld, int n
   if (!active_idx && n != ctx->cfg.seq_len) return MARCHE_EINVAL;
   if (is_new && !score_partial) return MARCHE_EINVAL;
   if (!ctx->bf16) return MARCHE_ESHAPE;
+  MARCHE_ENTER(ctx);
   if (n == 0) return MARCHE_OK;
   const marche_config& c = ctx->cfg;
   mark(ctx, MARCHE_KC_ATTENTION, (cudaStream_t)stream);
   MARCHE_TRY(launch_attention_twoseg(qkv, ld, c.width, 2 * c.width, c.batch, n, c.seq_len, c.n_heads, c.head_dim,
-                                     active_idx, cache_layer, is_new, score_partial, o, ctx->status_dev,
+                                     active_idx, cache_layer, is_new, score_partial, o, ctx->a_bf16, ctx->status_dev,
                                      (cudaStream_t)stream), "attention_twoseg");
   return MARCHE_OK;
 }
@@ -714,12 +769,14 @@ int marche_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void
   if (!ctx || !q || !cache_layer || !o || n < 0 || n > ctx->cfg.seq_len || ld_q < ctx->cfg.width)
     return MARCHE_EINVAL;
   if (is_new && !score_partial) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   return do_attention(ctx, q, ld_q, n, cache_layer, is_new, score_partial, o, (cudaStream_t)stream);
 }
 
 int marche_gather_rows(marche_ctx* ctx, const float* src, const int32_t* idx, int n, float* rows_out,
                        marche_stream stream) {
   if (!ctx || !src || !rows_out || n < 0 || n > ctx->cfg.seq_len || (n && !idx)) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   if (n == 0) return MARCHE_OK;
   mark(ctx, MARCHE_KC_OTHER, (cudaStream_t)stream);
   MARCHE_TRY(launch_gather_rows(src, idx, ctx->cfg.batch, n, ctx->cfg.seq_len, ctx->cfg.width, rows_out,
@@ -747,6 +804,7 @@ int marche_step_host(marche_ctx* ctx, int full, float* hidden, void* kv_cache, c
       (n_refresh_in && !refresh_in))
     return MARCHE_EINVAL;
   if (((uintptr_t)staging & 255) != 0) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   if (staging_bytes < marche_staging_bytes(ctx, max_new)) return MARCHE_EWORKSPACE;
   const size_t B = ctx->cfg.batch, D = ctx->cfg.width, mn = max_new;
   cudaStream_t st = (cudaStream_t)stream;
@@ -801,6 +859,7 @@ int marche_profile_begin(marche_ctx* ctx) {
 
 int marche_profile_end(marche_ctx* ctx, marche_stream stream, float* ms_per_class, int* launches_per_class) {
   if (!ctx || !ms_per_class || !launches_per_class) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);
   cudaStream_t st = (cudaStream_t)stream;
   const size_t n = ctx->event_class.size();
   mark(ctx, MARCHE_KC_OTHER, st);              // closing event
@@ -816,7 +875,7 @@ int marche_profile_end(marche_ctx* ctx, marche_stream stream, float* ms_per_clas
     ++launches_per_class[ctx->event_class[i]];
   }
   ctx->event_class.clear();
-  return MARCHE_OK;
+  return *(volatile int*)ctx->status_host ? MARCHE_ETIMEOUT : MARCHE_OK;
 }
 
 const char* marche_kernel_class_name(int cls) {
@@ -834,18 +893,15 @@ const char* marche_kernel_class_name(int cls) {
 static __device__ __align__(256) uint8_t g_static_mask_scratch[MARCHE_STATIC_SCRATCH_BYTES];
 
 namespace {
-constexpr int kMaxDevices = 64;
 uint8_t* g_static_mask_ptr[kMaxDevices] = {};
 
-// Device address of the scratch array on the current device (looked up on first use).
-cudaError_t static_mask_address(uint8_t** out) {
-  int dev = -1;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
+// Device address of the scratch array on device `dev`, which must be the current device (looked up on
+// first use: cudaGetSymbolAddress answers for the current device).
+cudaError_t static_mask_address(int dev, uint8_t** out) {
   if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
   if (!g_static_mask_ptr[dev]) {
     void* p = nullptr;
-    e = cudaGetSymbolAddress(&p, g_static_mask_scratch);
+    const cudaError_t e = cudaGetSymbolAddress(&p, g_static_mask_scratch);
     if (e != cudaSuccess) return e;
     g_static_mask_ptr[dev] = static_cast<uint8_t*>(p);
   }
@@ -858,9 +914,12 @@ int marche_select_refresh_static(marche_ctx* ctx, const float* scores, const int
                                  const int32_t* exclude_idx, int n_excl, int k, int32_t* refresh_idx,
                                  marche_stream stream) {
   if (!ctx || !scores || n_new < 0 || n_excl < 0 || k < 0) return MARCHE_EINVAL;
+  MARCHE_ENTER(ctx);                                   // the context's device is the current one from here on
   if ((n_new > 0 && !new_idx) || (n_excl > 0 && !exclude_idx)) return MARCHE_EINVAL;
   const int B = ctx->cfg.batch, S = ctx->cfg.seq_len;
   if (k > S - n_new - n_excl) return MARCHE_EINVAL;
+  if (k == 0) return MARCHE_OK;
+  if (!refresh_idx) return MARCHE_EINVAL;
   if ((size_t)B * (size_t)S > (size_t)MARCHE_STATIC_SCRATCH_BYTES) {
     char msg[160];
     snprintf(msg, sizeof msg, "marche_select_refresh_static: batch*seq_len = %zu exceeds the built-in scratch of %d bytes",
@@ -868,10 +927,8 @@ int marche_select_refresh_static(marche_ctx* ctx, const float* scores, const int
     ctx->last_error = msg;
     return MARCHE_EWORKSPACE;
   }
-  if (k == 0) return MARCHE_OK;
-  if (!refresh_idx) return MARCHE_EINVAL;
   uint8_t* mask = nullptr;
-  MARCHE_TRY(static_mask_address(&mask), "cudaGetSymbolAddress");
+  MARCHE_TRY(static_mask_address(ctx->device, &mask), "cudaGetSymbolAddress");
   cudaStream_t st = (cudaStream_t)stream;
   // The mask kernel writes all B*S bytes it uses, so nothing left over from an earlier call
   // (of this or any other context) can leak into this one.
@@ -879,6 +936,39 @@ int marche_select_refresh_static(marche_ctx* ctx, const float* scores, const int
   MARCHE_TRY(launch_step_flags(nullptr, 0, new_idx, n_new, exclude_idx, n_excl, B, S, nullptr, mask, st), "flags");
   mark(ctx, MARCHE_KC_TOPK, st);
   MARCHE_TRY(launch_topk(nullptr, 0, const_cast<float*>(scores), mask, B, S, k, refresh_idx, st), "topk");
+  return MARCHE_OK;
+}
+
+// ---------------------------------------------------------------- tuning, status, diagnostics
+int marche_get_tuning(const marche_ctx* ctx, marche_tuning* out) {
+  if (!ctx || !out) return MARCHE_EINVAL;
+  *out = ctx->tune;
+  return MARCHE_OK;
+}
+
+int marche_set_tuning(marche_ctx* ctx, const marche_tuning* t) {
+  if (!ctx || !t) return MARCHE_EINVAL;
+  if (t->attention_kernel < MARCHE_ATTENTION_AUTO || t->attention_kernel > MARCHE_ATTENTION_TCGEN05) return MARCHE_EINVAL;
+  if (t->gemm_kernel < MARCHE_GEMM_AUTO || t->gemm_kernel > MARCHE_GEMM_PAIR) return MARCHE_EINVAL;
+  if (t->tail_split != 0 && t->tail_split != 1 && t->tail_split != 2 && t->tail_split != 4) return MARCHE_EINVAL;
+  if (t->tile_n != 0 && t->tile_n != 128) return MARCHE_EINVAL;
+  if (t->attention_tc_min_rows < 0) return MARCHE_EINVAL;
+  ctx->tune = *t;
+  pdl_switch() = t->pdl != 0;
+  return MARCHE_OK;
+}
+
+int marche_check_status(marche_ctx* ctx, marche_stream stream) {
+  MARCHE_ENTER(ctx);
+  MARCHE_TRY(cudaStreamSynchronize((cudaStream_t)stream), "sync");
+  return *(volatile int*)ctx->status_host ? MARCHE_ETIMEOUT : MARCHE_OK;
+}
+
+int marche_debug_bounded_wait(marche_ctx* ctx, long long limit_cycles, marche_stream stream) {
+  MARCHE_ENTER(ctx);
+  if (limit_cycles < 1 || limit_cycles > 2000000000LL) return MARCHE_EINVAL;
+  mark(ctx, MARCHE_KC_OTHER, (cudaStream_t)stream);
+  MARCHE_TRY(launch_bounded_wait_probe(limit_cycles, ctx->status_dev, (cudaStream_t)stream), "bounded_wait_probe");
   return MARCHE_OK;
 }
 

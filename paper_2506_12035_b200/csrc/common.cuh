@@ -18,17 +18,23 @@ MARCHE_DEVINL float to_float(f16 v) { return __half2float(v); }
 template <typename T> MARCHE_DEVINL T from_float(float v);
 template <> MARCHE_DEVINL float from_float<float>(float v) { return v; }
 template <> MARCHE_DEVINL bf16 from_float<bf16>(float v) { return __float2bfloat16_rn(v); }
-template <> MARCHE_DEVINL f16 from_float<f16>(float v) { return __float2half_rn(v); }
 
 MARCHE_DEVINL uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&p);
 }
 
+// Two floats to packed IEEE fp16, round to nearest even, SATURATING: a magnitude beyond the largest
+// finite fp16 value becomes +-65504 instead of infinity (NaN stays NaN).  Every fp16 activation the
+// library writes (LayerNorm, attention and GELU outputs in the fp16-operand mode) goes through here.
 MARCHE_DEVINL uint32_t pack_f16x2(float lo, float hi) {
-  __half2 p = __floats2half2_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&p);
+  uint32_t r;
+  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
 }
+
+// Packed pair in the projections' operand type: bf16 when `bf`, saturating fp16 otherwise.
+MARCHE_DEVINL uint32_t pack_a16x2(float lo, float hi, bool bf) { return bf ? pack_bf16x2(lo, hi) : pack_f16x2(lo, hi); }
 
 MARCHE_DEVINL float2 unpack_bf16x2(uint32_t u) {
   __nv_bfloat162 p = *reinterpret_cast<__nv_bfloat162*>(&u);

@@ -5,7 +5,8 @@
 // to global memory (rows beyond M are clipped by the tensor map).
 //   EPI 0: out bf16 = acc + bias
 //   EPI 1: out fp32 += acc + bias   -- TMA reduce-add in L2, no read in the SM, one add per element
-//   EPI 2: out fp16 = GELU_erf(acc + bias)   (feeds the next projection as its A operand)
+//   EPI 2: out = GELU_erf(acc + bias) in the operand type, fp16 (saturating) or bf16 (feeds the next
+//          projection as its A operand)
 //   EPI 4: as EPI 0 for the q columns; the K and V columns go straight into scattered rows of the
 //          K/V cache (epilogue_box_scatter), so no separate write-back launch is needed
 #pragma once
@@ -20,7 +21,7 @@ namespace marche {
 // nullptr for EPI 1 (a partial sum of a split K range whose bias another piece adds).
 template <int EPI>
 MARCHE_DEVINL void epilogue_box(uint32_t t_addr, const float* __restrict__ bias_col, const CUtensorMap* out_map,
-                                int col, int row0, uint32_t stage, int lane) {
+                                int col, int row0, uint32_t stage, int lane, bool a_bf16) {
   // the previous box of this warp must have been read out of shared memory
   if (lane == 0) ptx::bulk_wait_read_all();
   __syncwarp();
@@ -57,7 +58,7 @@ MARCHE_DEVINL void epilogue_box(uint32_t t_addr, const float* __restrict__ bias_
         }
         const uint32_t dst = row_base + (uint32_t)(((hh * 4 + j) ^ (lane & 7)) << 4);
         uint32_t p0, p1, p2, p3;
-        if (EPI == 2) { p0 = pack_f16x2(v0, v1); p1 = pack_f16x2(v2, v3); p2 = pack_f16x2(v4, v5); p3 = pack_f16x2(v6, v7); }
+        if (EPI == 2) { p0 = pack_a16x2(v0, v1, a_bf16); p1 = pack_a16x2(v2, v3, a_bf16); p2 = pack_a16x2(v4, v5, a_bf16); p3 = pack_a16x2(v6, v7, a_bf16); }
         else { p0 = pack_bf16x2(v0, v1); p1 = pack_bf16x2(v2, v3); p2 = pack_bf16x2(v4, v5); p3 = pack_bf16x2(v6, v7); }
         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(p0), "r"(p1), "r"(p2), "r"(p3) : "memory");
       }

@@ -1,6 +1,6 @@
 // K1: index gather + LayerNorm (Algorithm 1 line 5, input side of the QKV and MLP
 // projections).  HBM-bound: each fp32 row is read once with 128-bit loads, kept in
-// registers for the two statistics passes, and written once as fp32 or fp16 (and, at block 0,
+// registers for the two statistics passes, and written once as fp32, fp16 or bf16 (and, at block 0,
 // once more as the compact fp32 residual row).
 //
 // One warp per row: lane l holds float4 number l, l+32, ... of the row (NV per lane),
@@ -87,13 +87,15 @@ static cudaError_t launch_ln_t(const float* src, int src_rows, const int32_t* id
   return err;
 }
 
-cudaError_t launch_gather_layernorm(bool half_out, const float* src, int src_rows, const int32_t* idx,
+cudaError_t launch_gather_layernorm(int out_kind, const float* src, int src_rows, const int32_t* idx,
                                     int B, int n, int D, const float* gamma, const float* beta, float eps,
                                     float* x_out, void* u_out, cudaStream_t st, const int32_t* out_idx,
                                     int out_rows) {
   if (D % 128 != 0) return cudaErrorInvalidValue;
-  if (half_out)
+  if (out_kind == OUT_F16)
     return launch_ln_t<f16>(src, src_rows, idx, B, n, D, gamma, beta, eps, x_out, (f16*)u_out, st, out_idx, out_rows);
+  if (out_kind == OUT_BF16)
+    return launch_ln_t<bf16>(src, src_rows, idx, B, n, D, gamma, beta, eps, x_out, (bf16*)u_out, st, out_idx, out_rows);
   return launch_ln_t<float>(src, src_rows, idx, B, n, D, gamma, beta, eps, x_out, (float*)u_out, st, out_idx, out_rows);
 }
 

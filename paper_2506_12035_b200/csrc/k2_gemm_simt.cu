@@ -1,10 +1,8 @@
 // K2 (SIMT): out = epilogue(a * w^T + bias) with fp32 FMA arithmetic.
 //
-// Operand types: fp32 x fp32, or (16-bit mode) fp16 activations x fp16 weights; the bias
-// epilogue writes T (fp32 / bf16: q, k, v), the GELU epilogue the activation type (fp32 / fp16).
-// This is the projection kernel of the fp32 configuration (the tensor cores have no
-// full-fp32 mode, and TF32 would not meet an fp32-level tolerance) and the bring-up
-// reference for the bf16 tensor-core kernel.  Classic shared-memory tiling: 64x64
+// fp32 operands and outputs only: this is the projection kernel of the fp32 configuration (the
+// tensor cores have no full-fp32 mode, and TF32 would not meet an fp32-level tolerance).  The
+// 16-bit contexts never come here.  Classic shared-memory tiling: 64x64
 // output tile, K step 16, 256 threads each owning a 4x4 micro-tile.
 #include "common.cuh"
 #include "kernels.h"
@@ -92,12 +90,11 @@ static cudaError_t launch_t(const TA* a, int lda, int M, const TA* w, const floa
   }
 }
 
-cudaError_t launch_gemm_simt(bool bf16_t, const void* a, int lda, int M, const void* w, const float* bias,
-                             int N, int K, int epilogue, void* out, cudaStream_t st) {
+cudaError_t launch_gemm_simt(const float* a, int lda, int M, const float* w, const float* bias,
+                             int N, int K, int epilogue, float* out, cudaStream_t st) {
   if (M == 0) return cudaSuccess;
   if (N % 64 || K % 16) return cudaErrorInvalidValue;
-  if (bf16_t) return launch_t<f16, bf16>((const f16*)a, lda, M, (const f16*)w, bias, N, K, epilogue, out, st);
-  return launch_t<float, float>((const float*)a, lda, M, (const float*)w, bias, N, K, epilogue, out, st);
+  return launch_t<float, float>(a, lda, M, w, bias, N, K, epilogue, out, st);
 }
 
 }  // namespace marche

@@ -1,7 +1,7 @@
 // K2: out = epilogue(a * w^T + bias) on the 5th-generation tensor cores.
 //
 // The QKV, output and MLP projections of the active rows (Algorithm 1 lines 5 and 9)
-// are dense 16-bit contractions (fp16 activations x fp16 weights -> fp32), so they run as a persistent, warp-specialised tcgen05
+// are dense 16-bit contractions (both operands fp16, or both bf16, -> fp32), so they run as a persistent, warp-specialised tcgen05
 // kernel: one CTA per SM walks over 128 x BN output tiles;
 //   warp 0   (one lane)  TMA producer: 128x64 A tile and BNx64 W tile per K step into a
 //                        shared-memory ring (128-byte swizzle), completion on mbarriers
@@ -47,7 +47,7 @@ template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                     const __grid_constant__ CUtensorMap tmap_out, int M, int N, int K,
-                    const float* __restrict__ bias, int* __restrict__ status) {
+                    const float* __restrict__ bias, int* __restrict__ status, int a_bf16) {
   using Cfg = GemmCfg<BN>;
   constexpr int STAGES = Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
@@ -123,7 +123,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = ptx::idesc_f16_f32(BM, BN);
+      const uint32_t idesc = ptx::idesc_16_f32(BM, BN, a_bf16 != 0);
       int it = 0, tile_i = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tile_i) {
@@ -168,7 +168,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
 #pragma unroll 1
         for (int c0 = 0; c0 < BN; c0 += EC)
           epilogue_box<EPI>(t_row + (uint32_t)c0, bias + n_blk * BN + c0, &tmap_out, n_blk * BN + c0, row0, my_stage,
-                            lane);
+                            lane, a_bf16 != 0);
       }
       ptx::tc_fence_before();
       __syncwarp();
@@ -200,14 +200,14 @@ int sm_count() { return device_sm_count(); }
 
 template <int BN, int EPI>
 cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& to, int M, int N, int K,
-                       const float* bias, int* status, cudaStream_t st) {
+                       const float* bias, int* status, int a_bf16, cudaStream_t st) {
   static size_t smem_set[kMaxDevices] = {};
   cudaError_t e = ensure_dynamic_smem(gemm_tcgen05_kernel<BN, EPI>, (size_t)GemmCfg<BN>::SMEM_BYTES, smem_set);
   if (e != cudaSuccess) return e;
   const int n_tiles = ((M + BM - 1) / BM) * (N / BN);
   const int grid = n_tiles < sm_count() ? n_tiles : sm_count();
   return launch_pdl(gemm_tcgen05_kernel<BN, EPI>, dim3(grid), dim3(kGemmThreads), (size_t)GemmCfg<BN>::SMEM_BYTES, st, ta,
-                    tw, to, M, N, K, bias, status);
+                    tw, to, M, N, K, bias, status, a_bf16);
 }
 
 }  // namespace
@@ -222,17 +222,17 @@ int gemm_tcgen05_pick_bn(int M, int N) {
 }
 
 cudaError_t launch_gemm_tcgen05(const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
-                                int epilogue, void* out, int* status, cudaStream_t st) {
+                                int epilogue, void* out, bool a_bf16, int* status, cudaStream_t st) {
   if (M == 0) return cudaSuccess;
   if (N % 128 || K % BK || lda % 8 || ((uintptr_t)a & 15) || ((uintptr_t)w & 15)) return cudaErrorInvalidValue;
   const int bn = gemm_tcgen05_pick_bn(M, N);
   CUtensorMap ta, tw, to;
-  if (!make_map_2d(&ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM, true)) return cudaErrorInvalidValue;
-  if (!make_map_2d(&tw, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)bn, true)) return cudaErrorInvalidValue;
+  if (!make_map_2d(&ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM, !a_bf16)) return cudaErrorInvalidValue;
+  if (!make_map_2d(&tw, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)bn, !a_bf16)) return cudaErrorInvalidValue;
   if (((uintptr_t)out & 15) || !tma_make_store_map(&to, out, (uint64_t)M, (uint64_t)N, epilogue == 1 ? 4 : 2))
     return cudaErrorInvalidValue;
 #define MARCHE_GEMM_CASE(BN_, EPI_) \
-  if (bn == BN_ && epilogue == EPI_) return launch_one<BN_, EPI_>(ta, tw, to, M, N, K, bias, status, st);
+  if (bn == BN_ && epilogue == EPI_) return launch_one<BN_, EPI_>(ta, tw, to, M, N, K, bias, status, a_bf16 ? 1 : 0, st);
   MARCHE_GEMM_CASE(256, 0) MARCHE_GEMM_CASE(256, 1) MARCHE_GEMM_CASE(256, 2)
   MARCHE_GEMM_CASE(128, 0) MARCHE_GEMM_CASE(128, 1) MARCHE_GEMM_CASE(128, 2)
 #undef MARCHE_GEMM_CASE

@@ -19,8 +19,6 @@
 // while its shared memory or TMEM can still be touched by the other.
 #include <cuda.h>
 
-#include <cstdlib>
-
 #include "gemm_epilogue.cuh"
 #include "kernels.h"
 #include "launch_pdl.h"
@@ -53,7 +51,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                          const __grid_constant__ CUtensorMap tmap_out, int M, int N, int K,
                          const float* __restrict__ bias, int* __restrict__ status, int* __restrict__ turn,
-                         const KvScatter kv, int tail_split) {
+                         const KvScatter kv, int tail_split, int a_bf16) {
   using Cfg = PairCfg<BN>;
   constexpr int STAGES = Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
@@ -206,7 +204,7 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       for (int i = 0; i < n_pieces && ok; ++i) {
         int tile, kb0, kb1, n_off, n_w;
         get_piece(i, tile, kb0, kb1, n_off, n_w);
-        const uint32_t idesc = ptx::idesc_f16_f32(2 * BM, n_w);
+        const uint32_t idesc = ptx::idesc_16_f32(2 * BM, n_w, a_bf16 != 0);
         const int acc = i & 1;
         const uint32_t acc_ph = (uint32_t)(i >> 1) & 1u;
         if (!ptx::mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -256,7 +254,7 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
               asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(my_turn) : "memory");
               if (v != 1 && (*abort_flag || clock64() - t0 > 2000000000LL)) { *abort_flag = 1; break; }
             } while (v != 1);
-            ptx::fence_proxy_async();
+            asm volatile("fence.proxy.async.global;" ::: "memory");   // the TMA reduce-adds below follow the acquire
           }
           __syncwarp();
           if (*abort_flag) { ok = false; break; }
@@ -287,7 +285,7 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
 #pragma unroll 1
           for (int c0 = c_begin; c0 < c_end; c0 += EC)
             epilogue_box<(EPI == 4) ? 0 : EPI>(t_row + (uint32_t)c0, bias_tile ? bias_tile + c0 : nullptr, &tmap_out,
-                                               col_tile + c0, row0, my_stage, lane);
+                                               col_tile + c0, row0, my_stage, lane, a_bf16 != 0);
         }
         if (my_turn && lane == 0) {
           if (kb0 == 0 && kb1 < n_kb) {
@@ -325,14 +323,52 @@ bool make_map_2d(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols
   return tma_make_map_bf16(map, ptr, 2, dims, strides, box, true, ieee_half);
 }
 
+// Number of CTA pairs of this kernel that can be resident at once on the current device (queried
+// once per device and instantiation).  The grid never exceeds it, so that every pair of a launch is
+// running while stream-K pieces wait for each other's turn flags.
+template <int BN, int EPI>
+cudaError_t max_resident_pairs(int* out) {
+  static int cached[kMaxDevices] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!cached[dev]) {
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * (sms / 2 > 0 ? sms / 2 : 1));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = (size_t)PairCfg<BN>::SMEM_BYTES;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    e = cudaOccupancyMaxActiveClusters(&clusters, gemm_tcgen05_2cta_kernel<BN, EPI>, &cfg);
+    if (e != cudaSuccess) return e;
+    if (clusters > sms / 2) clusters = sms / 2;
+    cached[dev] = clusters > 0 ? clusters : 1;
+  }
+  *out = cached[dev];
+  return cudaSuccess;
+}
+
 template <int BN, int EPI>
 cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& to, int M, int N, int K,
-                        const float* bias, int* status, int* turn, const KvScatter& kv, cudaStream_t st) {
+                        const float* bias, int* status, int* turn, const KvScatter& kv, int a_bf16, const GemmTuning& tune,
+                        cudaStream_t st) {
   static size_t smem_set[kMaxDevices] = {};
   cudaError_t e = ensure_dynamic_smem(gemm_tcgen05_2cta_kernel<BN, EPI>, (size_t)PairCfg<BN>::SMEM_BYTES, smem_set);
   if (e != cudaSuccess) return e;
   const int n_tiles = ((M + 2 * BM - 1) / (2 * BM)) * (N / BN);
-  const int max_pairs = device_sm_count() / 2;
+  int max_pairs = 1;
+  e = max_resident_pairs<BN, EPI>(&max_pairs);
+  if (e != cudaSuccess) return e;
   const int pairs = n_tiles < max_pairs ? n_tiles : max_pairs;
   // stream-K only for the reduce-add epilogue and only where whole tiles would waste a large part of
   // the last wave: a few waves at most (measured: +2 % on the cache-aware step, but -4 % on the
@@ -340,15 +376,11 @@ cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUte
   // ... and only for long tiles (K >= 2048, i.e. fc2): the completing piece has to wait until the first
   // piece's reduce-adds are complete, about 3 us after its last MMA, which a 16-K-block tile (7 us of MMA
   // work, the out-projection) cannot hide: measured 18 us with and without stream-K there.
-  int* use_turn = (EPI == 1 && turn && K >= 2048 && n_tiles > max_pairs && n_tiles % max_pairs != 0 &&
+  int* use_turn = (EPI == 1 && turn && tune.stream_k && K >= 2048 && n_tiles > max_pairs && n_tiles % max_pairs != 0 &&
                    n_tiles < 4 * max_pairs) ? turn : nullptr;
   // Whole-tile mode: cut the tiles of the last, partial round into 2 or 4 column slices when that
-  // shortens the round (cost model in tile units, below).  MARCHE_TAIL_SPLIT=0 turns it off.
-  static int split_on = -1;
-  if (split_on < 0) {
-    const char* e = getenv("MARCHE_TAIL_SPLIT");
-    split_on = e ? atoi(e) : 1;                      // 0 off, 1 cost model, 2 / 4 forced (measurement only)
-  }
+  // shortens the round (cost model in tile units, below).
+  const int split_on = tune.tail_split;              // 0 off, 1 cost model, 2 / 4 forced (measurement only)
   int tail_split = 1;
   const int left = n_tiles % pairs;
   if (!use_turn && (split_on == 2 || split_on == 4) && BN == 256 && left > 0) {
@@ -363,23 +395,18 @@ cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUte
     }
   }
   return launch_pdl(gemm_tcgen05_2cta_kernel<BN, EPI>, dim3(2 * pairs), dim3(kThreads), (size_t)PairCfg<BN>::SMEM_BYTES,
-                    st, ta, tw, to, M, N, K, bias, status, use_turn, kv, tail_split);
+                    st, ta, tw, to, M, N, K, bias, status, use_turn, kv, tail_split, a_bf16);
 }
 
 }  // namespace
 
 // Tile width: 256 whenever N allows it.  Measured on B200 at M = 4.3-5.8 k rows, the 128-wide
 // pair tile costs about 0.7x a 256-wide one (1.5x the operand bytes per flop), so it never wins
-// back what it gains in wave balance.  MARCHE_BN=128 overrides (measurement only).
-int gemm_tcgen05_2cta_pick_bn(int M, int N) {
-  static int forced = -1;
-  if (forced < 0) {
-    const char* e = getenv("MARCHE_BN");
-    forced = e ? atoi(e) : 0;
-  }
+// back what it gains in wave balance.  tile_n = 128 overrides (measurement only).
+int gemm_tcgen05_2cta_pick_bn(int M, int N, int tile_n) {
   (void)M;
   if (N % 256) return 128;
-  return forced == 128 ? 128 : 256;
+  return tile_n == 128 ? 128 : 256;
 }
 
 size_t gemm_tcgen05_2cta_turn_bytes(int M, int N) {
@@ -388,8 +415,8 @@ size_t gemm_tcgen05_2cta_turn_bytes(int M, int N) {
 }
 
 cudaError_t launch_gemm_tcgen05_2cta(const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
-                                     int epilogue, void* out, int* status, cudaStream_t st, int* turn,
-                                     const KvScatter* kv_scatter) {
+                                     int epilogue, void* out, bool a_bf16, int* status, cudaStream_t st,
+                                     const GemmTuning& tune, int* turn, const KvScatter* kv_scatter) {
   if (M == 0) return cudaSuccess;
   KvScatter kv = {nullptr, nullptr, 1, 1, 1, 1 << 30};
   if (epilogue == 4) {
@@ -400,14 +427,15 @@ cudaError_t launch_gemm_tcgen05_2cta(const void* a, int lda, int M, const void* 
     kv = *kv_scatter;
   }
   if (N % 128 || K % BK || lda % 8 || ((uintptr_t)a & 15) || ((uintptr_t)w & 15)) return cudaErrorInvalidValue;
-  const int bn = gemm_tcgen05_2cta_pick_bn(M, N);
+  const int bn = gemm_tcgen05_2cta_pick_bn(M, N, tune.tile_n);
   CUtensorMap ta, tw, to;
-  if (!make_map_2d(&ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM, true)) return cudaErrorInvalidValue;
-  if (!make_map_2d(&tw, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)(bn / 2), true)) return cudaErrorInvalidValue;
+  if (!make_map_2d(&ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM, !a_bf16)) return cudaErrorInvalidValue;
+  if (!make_map_2d(&tw, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)(bn / 2), !a_bf16)) return cudaErrorInvalidValue;
   if (((uintptr_t)out & 15) || !tma_make_store_map(&to, out, (uint64_t)M, (uint64_t)N, epilogue == 1 ? 4 : 2))
     return cudaErrorInvalidValue;
 #define MARCHE_GEMM2_CASE(BN_, EPI_) \
-  if (bn == BN_ && epilogue == EPI_) return launch_pair<BN_, EPI_>(ta, tw, to, M, N, K, bias, status, turn, kv, st);
+  if (bn == BN_ && epilogue == EPI_)   \
+    return launch_pair<BN_, EPI_>(ta, tw, to, M, N, K, bias, status, turn, kv, a_bf16 ? 1 : 0, tune, st);
   MARCHE_GEMM2_CASE(256, 0) MARCHE_GEMM2_CASE(256, 1) MARCHE_GEMM2_CASE(256, 2) MARCHE_GEMM2_CASE(256, 4)
   MARCHE_GEMM2_CASE(128, 0) MARCHE_GEMM2_CASE(128, 1) MARCHE_GEMM2_CASE(128, 2)
 #undef MARCHE_GEMM2_CASE

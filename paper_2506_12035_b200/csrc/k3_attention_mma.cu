@@ -12,7 +12,7 @@
 // several CTAs are resident per SM.  QK^T and PV
 // run on the tensor cores (mma.sync m16n8k16, bf16 in, fp32 accumulate; each warp owns
 // 16 query rows), softmax statistics stay in fp32 registers.  The output rows are written
-// as fp16: they are the A operand of the output projection.
+// in the projections' operand type (fp16 or bf16): they are the A operand of the output projection.
 //
 // Two flavours:
 //   plain    one pass, online softmax (running max / sum, rescaled accumulators);
@@ -36,20 +36,12 @@ namespace {
 
 using namespace att;
 
-// Optional fused write-back: k_off / v_off are the element offsets of the fresh K / V columns
-// relative to q (same row stride), idx the token of each row (nullptr = identity).
-struct WriteBack {
-  bf16* cache;            // nullptr: no write-back (the cache already holds the fresh rows)
-  const int32_t* idx;
-  int k_off, v_off;
-};
-
 // NWARPS consumer warps (16 query rows each) plus one producer warp.
 template <int DH, int NWARPS, bool SCORING>
 __global__ void __launch_bounds__((NWARPS + 1) * 32, NWARPS == 3 ? 4 : 1)
 attention_mma_kernel(const __grid_constant__ CUtensorMap tmap_kv, const bf16* __restrict__ q, int ld_q, int n,
                      int S, int H, int B, const uint8_t* __restrict__ is_new, float* __restrict__ score_partial,
-                     f16* __restrict__ o, int* __restrict__ status, WriteBack wb) {
+                     uint16_t* __restrict__ o, bool o_bf16, int* __restrict__ status) {
   using Cfg = AttCfg<DH>;
   constexpr int QT = NWARPS * 16;
   extern __shared__ uint8_t smem_raw[];
@@ -85,25 +77,6 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap tmap_kv, const bf16* __
     for (int t = threadIdx.x; t < NWARPS * S; t += (NWARPS + 1) * 32) colsum[t] = 0.f;
   __syncthreads();
   pdl_sync();                                          // set-up above overlaps the previous kernel's tail
-
-  if (wb.cache) {
-    // Fused cache write-back (Algorithm 1 line 11, done first so that the stream below sees the
-    // fresh rows): this CTA copies its head's K and V rows of the active tokens from the QKV
-    // projection's output into the cache.  No other CTA touches these columns.  The rows are
-    // then read back by TMA (async proxy), hence the cross-proxy fence before the barrier.
-    constexpr int CH = DH / 8;                         // 16-byte chunks per row
-    const size_t kv_stride = (size_t)B * S * H * DH;
-    for (int e = threadIdx.x; e < 2 * n * CH; e += (NWARPS + 1) * 32) {
-      const int which = e / (n * CH), r = e - which * n * CH;
-      const int j = r / CH, c = r - j * CH;
-      const int t = wb.idx ? wb.idx[(size_t)b * n + j] : j;
-      const uint4 v = *reinterpret_cast<const uint4*>(q + ((size_t)b * n + j) * ld_q + (which ? wb.v_off : wb.k_off) +
-                                                      h * DH + c * 8);
-      *reinterpret_cast<uint4*>(wb.cache + which * kv_stride + ((size_t)b * S + t) * (H * DH) + h * DH + c * 8) = v;
-    }
-    asm volatile("fence.proxy.async.global;" ::: "memory");
-    __syncthreads();
-  }
 
   bool ok = true;
   if (warp == NWARPS) {
@@ -302,12 +275,12 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap tmap_kv, const bf16* __
       if (warp_active && final_pass && kt == n_kv - 1) {
         const float f0 = SCORING ? 1.0f : 1.0f / l_run[0], f1 = SCORING ? 1.0f : 1.0f / l_run[1];
         const int r0 = qt * QT + warp * 16 + g, r1 = r0 + 8;
-        f16* o0 = o + ((size_t)b * n + r0) * D + h * DH + 2 * tg;
-        f16* o1 = o + ((size_t)b * n + r1) * D + h * DH + 2 * tg;
+        uint16_t* o0 = o + ((size_t)b * n + r0) * D + h * DH + 2 * tg;
+        uint16_t* o1 = o + ((size_t)b * n + r1) * D + h * DH + 2 * tg;
 #pragma unroll
         for (int j = 0; j < Cfg::ONT; ++j) {
-          if (r0 < n) *reinterpret_cast<uint32_t*>(o0 + 8 * j) = pack_f16x2(oacc[j][0] * f0, oacc[j][1] * f0);
-          if (r1 < n) *reinterpret_cast<uint32_t*>(o1 + 8 * j) = pack_f16x2(oacc[j][2] * f1, oacc[j][3] * f1);
+          if (r0 < n) *reinterpret_cast<uint32_t*>(o0 + 8 * j) = pack_a16x2(oacc[j][0] * f0, oacc[j][1] * f0, o_bf16);
+          if (r1 < n) *reinterpret_cast<uint32_t*>(o1 + 8 * j) = pack_a16x2(oacc[j][2] * f1, oacc[j][3] * f1, o_bf16);
         }
       }
     }
@@ -330,7 +303,7 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap tmap_kv, const bf16* __
 
 template <int DH, int NWARPS, bool SCORING>
 cudaError_t launch_att(const CUtensorMap& tm, const bf16* q, int ld_q, int B, int n, int S, int H,
-                       const uint8_t* is_new, float* partial, f16* o, int* status, WriteBack wb, cudaStream_t st) {
+                       const uint8_t* is_new, float* partial, uint16_t* o, bool o_bf16, int* status, cudaStream_t st) {
   const size_t smem = NSTAGE * AttCfg<DH>::STAGE_BYTES + 1024 + 64 + (SCORING ? (size_t)NWARPS * S * sizeof(float) : 0);
   static size_t smem_set[kMaxDevices] = {};
   cudaError_t e = ensure_dynamic_smem(attention_mma_kernel<DH, NWARPS, SCORING>, smem, smem_set);
@@ -338,19 +311,19 @@ cudaError_t launch_att(const CUtensorMap& tm, const bf16* q, int ld_q, int B, in
   // (Launching one sample's heads as a cluster, to co-schedule the CTAs that read neighbouring
   // 128-byte pieces of the same cache rows, was measured and does not help: 41.0 -> 41-43 us.)
   return launch_pdl(attention_mma_kernel<DH, NWARPS, SCORING>, dim3(B * H), dim3((NWARPS + 1) * 32), smem, st, tm, q, ld_q,
-                    n, S, H, B, is_new, partial, o, status, wb);
+                    n, S, H, B, is_new, partial, o, o_bf16, status);
 }
 
 template <int DH>
 cudaError_t launch_dh(const CUtensorMap& tm, const bf16* q, int ld_q, int B, int n, int S, int H,
-                      const uint8_t* is_new, float* partial, f16* o, int* status, WriteBack wb, cudaStream_t st) {
+                      const uint8_t* is_new, float* partial, uint16_t* o, bool o_bf16, int* status, cudaStream_t st) {
   const bool sc = is_new != nullptr;
   // 7 consumer warps + the producer warp = 256 threads: two CTAs per SM still fit the register file
   const int nw = n <= 16 ? 1 : (n <= 32 ? 2 : (n <= 48 ? 3 : (n <= 64 ? 4 : 7)));
 #define MARCHE_ATT_CASE(NW_)                                                                              \
   if (nw == NW_)                                                                                          \
-    return sc ? launch_att<DH, NW_, true>(tm, q, ld_q, B, n, S, H, is_new, partial, o, status, wb, st)     \
-              : launch_att<DH, NW_, false>(tm, q, ld_q, B, n, S, H, is_new, partial, o, status, wb, st);
+    return sc ? launch_att<DH, NW_, true>(tm, q, ld_q, B, n, S, H, is_new, partial, o, o_bf16, status, st) \
+              : launch_att<DH, NW_, false>(tm, q, ld_q, B, n, S, H, is_new, partial, o, o_bf16, status, st);
   MARCHE_ATT_CASE(1) MARCHE_ATT_CASE(2) MARCHE_ATT_CASE(3) MARCHE_ATT_CASE(4) MARCHE_ATT_CASE(7)
 #undef MARCHE_ATT_CASE
   return cudaErrorInvalidValue;
@@ -360,15 +333,8 @@ cudaError_t launch_dh(const CUtensorMap& tm, const bf16* q, int ld_q, int B, int
 
 cudaError_t launch_attention_mma(const void* q, int ld_q, int B, int n, int S, int H, int dh,
                                  const void* cache_layer, const uint8_t* is_new, float* score_partial, void* o,
-                                 int* status, cudaStream_t st, bool write_back, const int32_t* wb_idx, int k_off,
-                                 int v_off) {
+                                 bool o_bf16, int* status, cudaStream_t st) {
   if (n == 0) return cudaSuccess;
-  if (write_back && (ld_q % 8 || k_off % 8 || v_off % 8 || ((uintptr_t)q & 15))) return cudaErrorInvalidValue;
-  WriteBack wb;
-  wb.cache = write_back ? (bf16*)const_cast<void*>(cache_layer) : nullptr;
-  wb.idx = wb_idx;
-  wb.k_off = k_off;
-  wb.v_off = v_off;
   if ((dh != 64 && dh != 80) || ld_q % 2 || ((uintptr_t)q & 3) || ((uintptr_t)cache_layer & 15))
     return cudaErrorInvalidValue;
   const int D = H * dh;
@@ -378,8 +344,8 @@ cudaError_t launch_attention_mma(const void* q, int ld_q, int B, int n, int S, i
   const uint32_t box[3] = {(uint32_t)dh, KT, 1};
   if (!tma_make_map_bf16(&tm, cache_layer, 3, dims, strides, box, dh == 64)) return cudaErrorInvalidValue;
   if (dh == 64)
-    return launch_dh<64>(tm, (const bf16*)q, ld_q, B, n, S, H, is_new, score_partial, (f16*)o, status, wb, st);
-  return launch_dh<80>(tm, (const bf16*)q, ld_q, B, n, S, H, is_new, score_partial, (f16*)o, status, wb, st);
+    return launch_dh<64>(tm, (const bf16*)q, ld_q, B, n, S, H, is_new, score_partial, (uint16_t*)o, o_bf16, status, st);
+  return launch_dh<80>(tm, (const bf16*)q, ld_q, B, n, S, H, is_new, score_partial, (uint16_t*)o, o_bf16, status, st);
 }
 
 }  // namespace marche

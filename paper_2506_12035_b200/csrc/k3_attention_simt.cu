@@ -1,8 +1,7 @@
 // K3 (SIMT): attention of the active queries over all S cached rows of one block
 // (Algorithm 1 lines 6-8; by Appendix A this is plain softmax attention, Eq. 5, once
 // the active rows' fresh K, V are in the cache), with the relevance reduction of
-// Section 4.2 fused in.  fp32 arithmetic; serves the fp32 configuration and is the
-// bring-up reference for the tensor-core kernel.
+// Section 4.2 fused in.  fp32 arithmetic and storage; serves the fp32 configuration only.
 //
 // One CTA per (sample, head); warp w handles queries w, w+NW, ...  A query's whole
 // probability row lives in shared memory, so the softmax is the exact two-pass form
@@ -85,26 +84,17 @@ attention_simt_kernel(const T* __restrict__ q, int ld_q, int n, int S, int H, in
   }
 }
 
-cudaError_t launch_attention_simt(bool bf16_t, const void* q, int ld_q, int B, int n, int S, int H, int dh,
-                                  const void* cache_layer, const uint8_t* is_new, float* score_partial,
-                                  void* o, cudaStream_t st) {
+cudaError_t launch_attention_simt(const float* q, int ld_q, int B, int n, int S, int H, int dh,
+                                  const float* cache_layer, const uint8_t* is_new, float* score_partial,
+                                  float* o, cudaStream_t st) {
   if (n == 0) return cudaSuccess;
   const size_t smem = attention_simt_smem(S, dh);
   const long kv_stride = (long)B * S * H * dh;
-  cudaError_t e;
-  if (bf16_t) {
-    static size_t smem_set[kMaxDevices] = {};
-    e = ensure_dynamic_smem(attention_simt_kernel<bf16, f16>, smem, smem_set);
-    if (e != cudaSuccess) return e;
-    return launch_pdl(attention_simt_kernel<bf16, f16>, dim3(B * H), dim3(kAttWarps * 32), smem, st, (const bf16*)q, ld_q,
-                      n, S, H, dh, (const bf16*)cache_layer, kv_stride, is_new, score_partial, (f16*)o);
-  } else {
-    static size_t smem_set[kMaxDevices] = {};
-    e = ensure_dynamic_smem(attention_simt_kernel<float, float>, smem, smem_set);
-    if (e != cudaSuccess) return e;
-    return launch_pdl(attention_simt_kernel<float, float>, dim3(B * H), dim3(kAttWarps * 32), smem, st, (const float*)q,
-                      ld_q, n, S, H, dh, (const float*)cache_layer, kv_stride, is_new, score_partial, (float*)o);
-  }
+  static size_t smem_set[kMaxDevices] = {};
+  cudaError_t e = ensure_dynamic_smem(attention_simt_kernel<float, float>, smem, smem_set);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(attention_simt_kernel<float, float>, dim3(B * H), dim3(kAttWarps * 32), smem, st, q, ld_q, n, S, H, dh,
+                    cache_layer, kv_stride, is_new, score_partial, o);
 }
 
 }  // namespace marche

@@ -75,7 +75,8 @@ template <bool SCORING>
 __global__ void __launch_bounds__(kThreads)
 attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_constant__ CUtensorMap tmap_q,
                          int n, int S, int H, int B, const uint8_t* __restrict__ is_new,
-                         float* __restrict__ score_partial, f16* __restrict__ o, int* __restrict__ status) {
+                         float* __restrict__ score_partial, uint16_t* __restrict__ o, bool o_bf16,
+                         int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -338,19 +339,19 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __gr
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             uint4 v;
-            v.x = pack_f16x2(__uint_as_float(r0[8 * j + 0]) * inv, __uint_as_float(r0[8 * j + 1]) * inv);
-            v.y = pack_f16x2(__uint_as_float(r0[8 * j + 2]) * inv, __uint_as_float(r0[8 * j + 3]) * inv);
-            v.z = pack_f16x2(__uint_as_float(r0[8 * j + 4]) * inv, __uint_as_float(r0[8 * j + 5]) * inv);
-            v.w = pack_f16x2(__uint_as_float(r0[8 * j + 6]) * inv, __uint_as_float(r0[8 * j + 7]) * inv);
+            v.x = pack_a16x2(__uint_as_float(r0[8 * j + 0]) * inv, __uint_as_float(r0[8 * j + 1]) * inv, o_bf16);
+            v.y = pack_a16x2(__uint_as_float(r0[8 * j + 2]) * inv, __uint_as_float(r0[8 * j + 3]) * inv, o_bf16);
+            v.z = pack_a16x2(__uint_as_float(r0[8 * j + 4]) * inv, __uint_as_float(r0[8 * j + 5]) * inv, o_bf16);
+            v.w = pack_a16x2(__uint_as_float(r0[8 * j + 6]) * inv, __uint_as_float(r0[8 * j + 7]) * inv, o_bf16);
             dst[j] = v;
           }
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             uint4 v;
-            v.x = pack_f16x2(__uint_as_float(r1[8 * j + 0]) * inv, __uint_as_float(r1[8 * j + 1]) * inv);
-            v.y = pack_f16x2(__uint_as_float(r1[8 * j + 2]) * inv, __uint_as_float(r1[8 * j + 3]) * inv);
-            v.z = pack_f16x2(__uint_as_float(r1[8 * j + 4]) * inv, __uint_as_float(r1[8 * j + 5]) * inv);
-            v.w = pack_f16x2(__uint_as_float(r1[8 * j + 6]) * inv, __uint_as_float(r1[8 * j + 7]) * inv);
+            v.x = pack_a16x2(__uint_as_float(r1[8 * j + 0]) * inv, __uint_as_float(r1[8 * j + 1]) * inv, o_bf16);
+            v.y = pack_a16x2(__uint_as_float(r1[8 * j + 2]) * inv, __uint_as_float(r1[8 * j + 3]) * inv, o_bf16);
+            v.z = pack_a16x2(__uint_as_float(r1[8 * j + 4]) * inv, __uint_as_float(r1[8 * j + 5]) * inv, o_bf16);
+            v.w = pack_a16x2(__uint_as_float(r1[8 * j + 6]) * inv, __uint_as_float(r1[8 * j + 7]) * inv, o_bf16);
             dst[4 + j] = v;
           }
         }
@@ -374,20 +375,20 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __gr
 
 template <bool SCORING>
 cudaError_t launch_tc(const CUtensorMap& tkv, const CUtensorMap& tq, int B, int n, int S, int H, const uint8_t* is_new,
-                      float* partial, f16* o, int* status, cudaStream_t st) {
+                      float* partial, uint16_t* o, bool o_bf16, int* status, cudaStream_t st) {
   const size_t smem = SMEM_FIXED + (SCORING ? (size_t)4 * S * sizeof(float) : 0);
   static size_t smem_set[kMaxDevices] = {};
   cudaError_t e = ensure_dynamic_smem(attention_tcgen05_kernel<SCORING>, smem, smem_set);
   if (e != cudaSuccess) return e;
   return launch_pdl(attention_tcgen05_kernel<SCORING>, dim3(B * H), dim3(kThreads), smem, st, tkv, tq, n, S, H, B, is_new,
-                    partial, o, status);
+                    partial, o, o_bf16, status);
 }
 
 }  // namespace
 
 cudaError_t launch_attention_tcgen05(const void* q, int ld_q, int B, int n, int S, int H, int dh,
                                      const void* cache_layer, const uint8_t* is_new, float* score_partial, void* o,
-                                     int* status, cudaStream_t st) {
+                                     bool o_bf16, int* status, cudaStream_t st) {
   if (n == 0) return cudaSuccess;
   if (dh != DH || ld_q % 8 || ((uintptr_t)q & 15) || ((uintptr_t)cache_layer & 15) || S > 2048)
     return cudaErrorInvalidValue;
@@ -405,8 +406,8 @@ cudaError_t launch_attention_tcgen05(const void* q, int ld_q, int B, int n, int 
     const uint32_t box[3] = {(uint32_t)DH, QT, 1};
     if (!tma_make_map_bf16(&tq, q, 3, dims, strides, box, true)) return cudaErrorInvalidValue;
   }
-  return is_new ? launch_tc<true>(tkv, tq, B, n, S, H, is_new, score_partial, (f16*)o, status, st)
-                : launch_tc<false>(tkv, tq, B, n, S, H, is_new, score_partial, (f16*)o, status, st);
+  return is_new ? launch_tc<true>(tkv, tq, B, n, S, H, is_new, score_partial, (uint16_t*)o, o_bf16, status, st)
+                : launch_tc<false>(tkv, tq, B, n, S, H, is_new, score_partial, (uint16_t*)o, o_bf16, status, st);
 }
 
 }  // namespace marche

@@ -31,7 +31,7 @@ attention_twoseg_kernel(const __grid_constant__ CUtensorMap tmap_c, const __grid
                         const bf16* __restrict__ qkv, int ld, int k_off, int v_off, int n, int S, int H, int B,
                         const int32_t* __restrict__ active_idx, bf16* __restrict__ cache_layer,
                         const uint8_t* __restrict__ is_new, float* __restrict__ score_partial,
-                        f16* __restrict__ o, int* __restrict__ status) {
+                        uint16_t* __restrict__ o, bool o_bf16, int* __restrict__ status) {
   using Cfg = AttCfg<DH>;
   constexpr int QT = NWARPS * 16;
   constexpr int NTHREADS = (NWARPS + 1) * 32;
@@ -301,12 +301,12 @@ attention_twoseg_kernel(const __grid_constant__ CUtensorMap tmap_c, const __grid
       if (warp_active && final_pass && u == n_t - 1) {
         const float f0 = SCORING ? 1.0f : 1.0f / l_run[0], f1 = SCORING ? 1.0f : 1.0f / l_run[1];
         const int r0 = qt * QT + warp * 16 + g, r1 = r0 + 8;
-        f16* o0 = o + ((size_t)b * n + r0) * D + h * DH + 2 * tg;
-        f16* o1 = o + ((size_t)b * n + r1) * D + h * DH + 2 * tg;
+        uint16_t* o0 = o + ((size_t)b * n + r0) * D + h * DH + 2 * tg;
+        uint16_t* o1 = o + ((size_t)b * n + r1) * D + h * DH + 2 * tg;
 #pragma unroll
         for (int j = 0; j < Cfg::ONT; ++j) {
-          if (r0 < n) *reinterpret_cast<uint32_t*>(o0 + 8 * j) = pack_f16x2(oacc[j][0] * f0, oacc[j][1] * f0);
-          if (r1 < n) *reinterpret_cast<uint32_t*>(o1 + 8 * j) = pack_f16x2(oacc[j][2] * f1, oacc[j][3] * f1);
+          if (r0 < n) *reinterpret_cast<uint32_t*>(o0 + 8 * j) = pack_a16x2(oacc[j][0] * f0, oacc[j][1] * f0, o_bf16);
+          if (r1 < n) *reinterpret_cast<uint32_t*>(o1 + 8 * j) = pack_a16x2(oacc[j][2] * f1, oacc[j][3] * f1, o_bf16);
         }
       }
     }
@@ -339,28 +339,28 @@ attention_twoseg_kernel(const __grid_constant__ CUtensorMap tmap_c, const __grid
 template <int DH, int NWARPS, bool SCORING>
 cudaError_t launch_ts(const CUtensorMap& tc, const CUtensorMap& ta, const bf16* qkv, int ld, int k_off, int v_off,
                       int B, int n, int S, int H, const int32_t* idx, bf16* cache, const uint8_t* is_new,
-                      float* partial, f16* o, int* status, cudaStream_t st) {
+                      float* partial, uint16_t* o, bool o_bf16, int* status, cudaStream_t st) {
   const size_t smem = NSTAGE * AttCfg<DH>::STAGE_BYTES + 1024 + 64 + 32 * 8 + 32 + (((size_t)n * 4 + 15) & ~(size_t)15) +
                       (SCORING ? (size_t)NWARPS * S * sizeof(float) : 0);
   static size_t smem_set[kMaxDevices] = {};
   cudaError_t e = ensure_dynamic_smem(attention_twoseg_kernel<DH, NWARPS, SCORING>, smem, smem_set);
   if (e != cudaSuccess) return e;
   return launch_pdl(attention_twoseg_kernel<DH, NWARPS, SCORING>, dim3(B * H), dim3((NWARPS + 1) * 32), smem, st, tc, ta,
-                    qkv, ld, k_off, v_off, n, S, H, B, idx, cache, is_new, partial, o, status);
+                    qkv, ld, k_off, v_off, n, S, H, B, idx, cache, is_new, partial, o, o_bf16, status);
 }
 
 template <int DH>
 cudaError_t launch_ts_dh(const CUtensorMap& tc, const CUtensorMap& ta, const bf16* qkv, int ld, int k_off, int v_off,
                          int B, int n, int S, int H, const int32_t* idx, bf16* cache, const uint8_t* is_new,
-                         float* partial, f16* o, int* status, cudaStream_t st) {
+                         float* partial, uint16_t* o, bool o_bf16, int* status, cudaStream_t st) {
   const bool sc = is_new != nullptr;
   const int nw = n <= 16 ? 1 : (n <= 32 ? 2 : (n <= 48 ? 3 : (n <= 64 ? 4 : 7)));
 #define MARCHE_TS_CASE(NW_)                                                                                          \
   if (nw == NW_)                                                                                                     \
     return sc ? launch_ts<DH, NW_, true>(tc, ta, qkv, ld, k_off, v_off, B, n, S, H, idx, cache, is_new, partial, o,   \
-                                         status, st)                                                                 \
+                                         o_bf16, status, st)                                                         \
               : launch_ts<DH, NW_, false>(tc, ta, qkv, ld, k_off, v_off, B, n, S, H, idx, cache, is_new, partial, o,  \
-                                          status, st);
+                                          o_bf16, status, st);
   MARCHE_TS_CASE(1) MARCHE_TS_CASE(2) MARCHE_TS_CASE(3) MARCHE_TS_CASE(4) MARCHE_TS_CASE(7)
 #undef MARCHE_TS_CASE
   return cudaErrorInvalidValue;
@@ -370,7 +370,7 @@ cudaError_t launch_ts_dh(const CUtensorMap& tc, const CUtensorMap& ta, const bf1
 
 cudaError_t launch_attention_twoseg(const void* qkv, int ld, int k_off, int v_off, int B, int n, int S, int H, int dh,
                                     const int32_t* active_idx, void* cache_layer, const uint8_t* is_new,
-                                    float* score_partial, void* o, int* status, cudaStream_t st) {
+                                    float* score_partial, void* o, bool o_bf16, int* status, cudaStream_t st) {
   if (n == 0) return cudaSuccess;
   if ((dh != 64 && dh != 80) || ld % 8 || k_off % 8 || v_off % 8 || ((uintptr_t)qkv & 15) ||
       ((uintptr_t)cache_layer & 15) || S > 2048 || n > S)
@@ -391,9 +391,9 @@ cudaError_t launch_attention_twoseg(const void* qkv, int ld, int k_off, int v_of
   }
   if (dh == 64)
     return launch_ts_dh<64>(tc, ta, (const bf16*)qkv, ld, k_off, v_off, B, n, S, H, active_idx, (bf16*)cache_layer, is_new,
-                            score_partial, (f16*)o, status, st);
+                            score_partial, (uint16_t*)o, o_bf16, status, st);
   return launch_ts_dh<80>(tc, ta, (const bf16*)qkv, ld, k_off, v_off, B, n, S, H, active_idx, (bf16*)cache_layer, is_new,
-                          score_partial, (f16*)o, status, st);
+                          score_partial, (uint16_t*)o, o_bf16, status, st);
 }
 
 }  // namespace marche

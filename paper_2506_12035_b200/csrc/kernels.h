@@ -8,8 +8,11 @@
 
 namespace marche {
 
-// K1: gather + LayerNorm (output fp16 when half_out, else fp32).  rows = B*n; src row of (b, j) is src[b][idx ? idx[b][j] : j].
-cudaError_t launch_gather_layernorm(bool half_out, const float* src, int src_rows, const int32_t* idx,
+// Element type of an activation output: fp32, saturating IEEE fp16, or bf16.
+enum { OUT_F32 = 0, OUT_F16 = 1, OUT_BF16 = 2 };
+
+// K1: gather + LayerNorm (output type out_kind).  rows = B*n; src row of (b, j) is src[b][idx ? idx[b][j] : j].
+cudaError_t launch_gather_layernorm(int out_kind, const float* src, int src_rows, const int32_t* idx,
                                     int B, int n, int D, const float* gamma, const float* beta, float eps,
                                     float* x_out, void* u_out, cudaStream_t st, const int32_t* out_idx = nullptr,
                                     int out_rows = 0);
@@ -52,14 +55,15 @@ cudaError_t launch_validate(const int32_t* active_idx, int n_active, const int32
 cudaError_t launch_topk(const float* partial, int H, float* scores, const uint8_t* cand, int B, int S, int k,
                         int32_t* refresh_idx, cudaStream_t st, int policy = 0, uint32_t seed = 0);
 
-// K2 (fp32 SIMT and bf16 SIMT bring-up path).
-cudaError_t launch_gemm_simt(bool bf16_t, const void* a, int lda, int M, const void* w, const float* bias,
-                             int N, int K, int epilogue, void* out, cudaStream_t st);
+// K2 of the fp32 configuration (SIMT, fp32 operands and outputs).
+cudaError_t launch_gemm_simt(const float* a, int lda, int M, const float* w, const float* bias,
+                             int N, int K, int epilogue, float* out, cudaStream_t st);
 
-// K2 (bf16, tcgen05/TMEM fed by TMA).  N % 128 == 0, K % 64 == 0, lda % 8 == 0, 16-byte aligned
-// operands.  `status` is a device-visible int that bounded waits set when they give up.
+// K2 (16-bit operands, tcgen05/TMEM fed by TMA).  N % 128 == 0, K % 64 == 0, lda % 8 == 0, 16-byte aligned
+// operands.  a_bf16: both operands (and the GELU epilogue's output) are bf16, otherwise IEEE fp16.
+// `status` is a device-visible int that bounded waits set when they give up.
 cudaError_t launch_gemm_tcgen05(const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
-                                int epilogue, void* out, int* status, cudaStream_t st);
+                                int epilogue, void* out, bool a_bf16, int* status, cudaStream_t st);
 int gemm_tcgen05_pick_bn(int M, int N);
 // Where the K and V columns of a fused QKV projection go (Algorithm 1 line 11 done by the projection's
 // epilogue, epilogue code 4): row r of the GEMM is active token j = r % n of sample b = r / n, its cache row is
@@ -74,39 +78,46 @@ struct KvScatter {
 // Same contract, tcgen05.mma cta_group::2: CTA pairs share 256 x BN tiles (cluster of 2, no multicast).
 // `turn`: optional zero-filled device scratch of gemm_tcgen05_2cta_turn_bytes(M, N) bytes; with it the
 // residual epilogue may use stream-K (ordered reduce-adds; the flags are left zero again).
+struct GemmTuning {
+  bool stream_k = true;   // residual epilogue: stream-K with ordered reduce-adds where it pays
+  int tail_split = 1;     // partial last round of tiles cut into column slices: 0 off, 1 cost model, 2 / 4 forced
+  int tile_n = 0;         // 0: 256-wide tiles whenever N allows; 128 forces the narrow tile
+};
 cudaError_t launch_gemm_tcgen05_2cta(const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
-                                     int epilogue, void* out, int* status, cudaStream_t st, int* turn = nullptr,
+                                     int epilogue, void* out, bool a_bf16, int* status, cudaStream_t st,
+                                     const GemmTuning& tune, int* turn = nullptr,
                                      const KvScatter* kv_scatter = nullptr);
 size_t gemm_tcgen05_2cta_turn_bytes(int M, int N);
-int gemm_tcgen05_2cta_pick_bn(int M, int N);
+int gemm_tcgen05_2cta_pick_bn(int M, int N, int tile_n);
 
-// K3 (SIMT): attention of n queries per sample over all S cache rows.
-cudaError_t launch_attention_simt(bool bf16_t, const void* q, int ld_q, int B, int n, int S, int H, int dh,
-                                  const void* cache_layer, const uint8_t* is_new, float* score_partial,
-                                  void* o, cudaStream_t st);
+// K3 of the fp32 configuration (SIMT): attention of n queries per sample over all S cache rows.
+cudaError_t launch_attention_simt(const float* q, int ld_q, int B, int n, int S, int H, int dh,
+                                  const float* cache_layer, const uint8_t* is_new, float* score_partial,
+                                  float* o, cudaStream_t st);
 size_t attention_simt_smem(int S, int dh);
 
-// K3 (bf16, TMA-staged K/V tiles, tensor-core QK^T and PV, fused score column sums).
-// head_dim 64 or 80; ld_q even; cache_layer 16-byte aligned.
-// write_back: each CTA first copies its head's fresh K / V rows (columns k_off / v_off relative to q,
-// same row stride; token of row j = wb_idx[b][j], nullptr = identity) into cache_layer, replacing a
-// separate launch_scatter_kv (needs ld_q % 8 == 0 and q 16-byte aligned).
+// K3 (bf16 q / cache, TMA-staged K/V tiles, tensor-core QK^T and PV, fused score column sums).
+// head_dim 64 or 80; ld_q even; cache_layer 16-byte aligned.  o is written in the projections'
+// operand type: bf16 when o_bf16, saturating fp16 otherwise.
 cudaError_t launch_attention_mma(const void* q, int ld_q, int B, int n, int S, int H, int dh,
                                  const void* cache_layer, const uint8_t* is_new, float* score_partial, void* o,
-                                 int* status, cudaStream_t st, bool write_back = false, const int32_t* wb_idx = nullptr,
-                                 int k_off = 0, int v_off = 0);
+                                 bool o_bf16, int* status, cudaStream_t st);
 
 // K3 on tcgen05 (head_dim 64 only): S = Q K^T and O = P V as tcgen05.mma with TMEM accumulators.
 // ld_q % 8 == 0; q and cache_layer 16-byte aligned.
 cudaError_t launch_attention_tcgen05(const void* q, int ld_q, int B, int n, int S, int H, int dh,
                                      const void* cache_layer, const uint8_t* is_new, float* score_partial, void* o,
-                                     int* status, cudaStream_t st);
+                                     bool o_bf16, int* status, cudaStream_t st);
 
 // K3, two-segment flavour (Eq. 6-10 without concatenation, then the cache write-back of Algorithm 1
 // line 11 by the same kernel): fresh K/V are columns k_off / v_off of the compact qkv buffer
 // [B*n][ld]; active_idx NULL = identity.  Same type and alignment rules as launch_attention_mma.
 cudaError_t launch_attention_twoseg(const void* qkv, int ld, int k_off, int v_off, int B, int n, int S, int H, int dh,
                                     const int32_t* active_idx, void* cache_layer, const uint8_t* is_new,
-                                    float* score_partial, void* o, int* status, cudaStream_t st);
+                                    float* score_partial, void* o, bool o_bf16, int* status, cudaStream_t st);
+
+// Diagnostic: one thread waits, with the library's bounded mbarrier wait, on a barrier nothing ever
+// arrives on; after limit_cycles it gives up, writes a code to *status and the kernel returns.
+cudaError_t launch_bounded_wait_probe(long long limit_cycles, int* status, cudaStream_t st);
 
 }  // namespace marche

@@ -202,11 +202,12 @@ MARCHE_DEVINL uint64_t smem_desc_k_sw128(uint32_t addr) {
   return ((uint64_t)hi << 32) | lo;
 }
 
-// Instruction descriptor of tcgen05.mma kind::f16 with fp32 D (c_format 1), both operands K-major
-// IEEE fp16 (a_format = b_format = 0; the two formats must be equal: a mixed fp16 x bf16
-// descriptor is rejected by the hardware as an illegal instruction).
-MARCHE_DEVINL constexpr uint32_t idesc_f16_f32(int M, int N) {
-  return (1u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+// Instruction descriptor of tcgen05.mma kind::f16 with fp32 D (c_format 1), both operands K-major and
+// of the same 16-bit format: IEEE fp16 (a_format = b_format = 0) or bf16 (1).  The two formats must be
+// equal: a mixed fp16 x bf16 descriptor is rejected by the hardware as an illegal instruction.
+MARCHE_DEVINL constexpr uint32_t idesc_16_f32(int M, int N, bool bf) {
+  return (1u << 4) | ((bf ? 1u : 0u) << 7) | ((bf ? 1u : 0u) << 10) | ((uint32_t)(N >> 3) << 17) |
+         ((uint32_t)(M >> 4) << 24);
 }
 
 }  // namespace ptx

@@ -17,9 +17,10 @@ from helpers import TOL, dev, idx_dev, make_model, max_abs, rel_l2
 pytestmark = pytest.mark.gpu
 
 
-def _sampled_parity(cfg, ratio, n_steps=3, also_full_recompute=False):
+def _sampled_parity(cfg, ratio, n_steps=3, also_full_recompute=False, operand="f16", bound=None):
     """GPU on the whole batch against the oracle on the first and the last guidance pair
     (rows 0, B/2 and B/2-1, B-1: the last rows sit in the clipped tail tile of every projection).
+    `bound` replaces the acceptance bound on hidden rows and cache (index work stays bit-exact).
     Returns the largest max-abs seen on the hidden rows."""
     if torch.cuda.get_device_properties(0).total_memory < 40e9:
         pytest.skip("needs a large GPU")
@@ -27,7 +28,7 @@ def _sampled_parity(cfg, ratio, n_steps=3, also_full_recompute=False):
     rows_s = [0, half, half - 1, cfg.B - 1]            # sampled batch rows
     ratio = float(np.float32(ratio))                   # the C ABI takes a float
     blocks = synth.make_weights(cfg)
-    m = make_model(cfg, blocks)
+    m = make_model(cfg, blocks, operand=operand)
     hidden_np = synth.make_hidden(cfg)
     sets = synth.new_token_sets(cfg, synth.generation_orders(cfg))
 
@@ -64,7 +65,7 @@ def _sampled_parity(cfg, ratio, n_steps=3, also_full_recompute=False):
     m.init_cache(cache)
     refresh = torch.zeros(B * S, dtype=torch.int32, device="cuda")
     scores = torch.empty(B, S, device="cuda")
-    ma, rl = TOL["bf16"]
+    ma, rl = TOL["bf16"] if bound is None else bound
     k_prev = 0
     worst = 0.0
     for t in range(n_steps):
@@ -129,7 +130,8 @@ def _sampled_parity(cfg, ratio, n_steps=3, also_full_recompute=False):
         dk = float((cache_f.float() - cache.float()).abs().max())
         print("all-active step vs full step on the device: hidden max-abs %.3g, cache max-abs %.3g" % (d, dk))
         assert d <= ma / 3 and dk <= ma / 3
-    print("full-size parity %s ratio %.2f: hidden max-abs %.3g, cache K max-abs %.3g" % (cfg.name, ratio, worst, max_abs(Kc, cache2.K)))
+    print("full-size parity %s ratio %.2f, %s operands: hidden max-abs %.3g, cache K max-abs %.3g"
+          % (cfg.name, ratio, operand, worst, max_abs(Kc, cache2.K)))
     return worst
 
 
@@ -145,6 +147,17 @@ def test_full_size_refresh_ratio_sweep(ratio):
     variants), 5 %, 20 % (66..77 tokens) and 100 %, where every token is active in a permuted order and the
     step must equal the full recompute (Appendix A)."""
     _sampled_parity(synth.CONFIGS["mar_l"], ratio, also_full_recompute=(ratio == 1.0))
+
+
+def test_full_size_all_bf16_operands_recorded(record_property):
+    """The MAR-L stack with bf16 projection operands (MARCHE_BF16), all 32 blocks: the rounding of the
+    LayerNorm / attention / GELU outputs to bf16 puts the hidden rows outside the 3e-2 bound that the fp16
+    operand mode meets, which is why that mode exists.  The figure is recorded, not gated: the test only
+    requires that the path runs, stays within a loose sanity bound and keeps its index work exact."""
+    cfg = synth.CONFIGS["mar_l"]
+    worst = _sampled_parity(cfg, cfg.ratio, operand="bf16", bound=(0.25, 3e-2))
+    record_property("all_bf16_hidden_max_abs", worst)
+    print("MAR-L, bf16 operands throughout: hidden max-abs %.3g (acceptance bound of the fp16-operand mode: 3e-2)" % worst)
 
 
 def test_full_size_high_resolution_256_steps():

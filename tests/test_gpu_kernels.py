@@ -14,32 +14,41 @@ pytestmark = pytest.mark.gpu
 
 
 def model_for(dtype, D, H, F, S, B, L=1):
-    cfg = synth.CONFIGS["tiny"].replace(L=L, E=0, D=D, H=H, F=F, S=S, B=B, dtype=dtype, n_buffer=0)
+    """dtype "f32", "bf16" (bf16 cache, fp16 projection operands) or "bf16b" (bf16 throughout)."""
+    cfg = synth.CONFIGS["tiny"].replace(L=L, E=0, D=D, H=H, F=F, S=S, B=B, dtype="f32" if dtype == "f32" else "bf16",
+                                        n_buffer=0)
     blocks = synth.make_weights(cfg)
-    return cfg, blocks, make_model(cfg, blocks)
+    return cfg, blocks, make_model(cfg, blocks, operand="bf16" if dtype == "bf16b" else "f16")
 
 
 def tdt(dtype):
-    """element type of weights, q/k/v and the K/V cache"""
-    return torch.bfloat16 if dtype == "bf16" else torch.float32
+    """element type of q/k/v and the K/V cache"""
+    return torch.float32 if dtype == "f32" else torch.bfloat16
 
 
 def adt(dtype):
-    """element type of the activation matrices that feed a projection (fp16 in 16-bit mode)"""
-    return torch.float16 if dtype == "bf16" else torch.float32
+    """element type of the projections' operands: weight matrices and the activations that feed them"""
+    return {"f32": torch.float32, "bf16": torch.float16, "bf16b": torch.bfloat16}[dtype]
 
 
 def quant_a(a, dtype):
-    return np.asarray(a, np.float32).astype(np.float16).astype(np.float64) if dtype == "bf16" else np.asarray(a, np.float32).astype(np.float64)
+    """What the device holds for a projection operand."""
+    a = np.asarray(a, np.float32)
+    if dtype == "bf16":
+        return a.astype(np.float16).astype(np.float64)
+    return synth.round_to_bf16(a).astype(np.float64) if dtype == "bf16b" else a.astype(np.float64)
 
 
 def quant(a, dtype):
-    """What the device holds for an operand of the compute type."""
-    return synth.round_to_bf16(a).astype(np.float64) if dtype == "bf16" else np.asarray(a, np.float32).astype(np.float64)
+    """What the device holds for q/k/v and cache entries."""
+    return np.asarray(a, np.float32).astype(np.float64) if dtype == "f32" else synth.round_to_bf16(a).astype(np.float64)
+
+
+LOW = ("bf16", "bf16b")        # the 16-bit contexts
 
 
 # ------------------------------------------------------------------ K1 gather + LayerNorm
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "bf16b"])
 @pytest.mark.parametrize("D,H", [(256, 4), (768, 12), (1024, 16), (1280, 16)])
 @pytest.mark.parametrize("n", [1, 2, 41, 68])
 def test_gather_layernorm(dtype, D, H, n):
@@ -58,17 +67,17 @@ def test_gather_layernorm(dtype, D, H, n):
         X = np.stack([hidden[b, idx[b]] for b in range(B)]).reshape(B * n, D)
         assert np.array_equal(x_out.cpu().numpy(), X)                       # the gather is a copy: exact
         want = orc.layer_norm(X.astype(np.float64), g.astype(np.float64), be.astype(np.float64), cfg.ln_eps)
-        assert_close(host(u_out), want, dtype, "LN", scale=1.0 if dtype == "bf16" else 10.0)
+        assert_close(host(u_out), want, dtype, "LN", scale=1.0 if dtype in LOW else 10.0)
     # identity index (idx NULL), no compact copy
     u_out = torch.zeros(B * n, D, dtype=adt(dtype), device="cuda")
     m.gather_layernorm(dev(hidden), None, n, dev(g), dev(be), None, u_out)
     want = orc.layer_norm(hidden[:, :n].reshape(B * n, D).astype(np.float64), g.astype(np.float64),
                           be.astype(np.float64), cfg.ln_eps)
-    assert_close(host(u_out), want, dtype, "LN identity", scale=1.0 if dtype == "bf16" else 10.0)
+    assert_close(host(u_out), want, dtype, "LN identity", scale=1.0 if dtype in LOW else 10.0)
 
 
 # ------------------------------------------------------------------ K2 projections
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "bf16b"])
 @pytest.mark.parametrize("M", [1, 24, 62, 129, 300])
 @pytest.mark.parametrize("N,K", [(768, 256), (256, 256), (1024, 256), (256, 1024), (384, 128), (128, 320)])
 def test_linear_all_epilogues(dtype, M, N, K):
@@ -84,8 +93,8 @@ def test_linear_all_epilogues(dtype, M, N, K):
     # bias
     out = torch.zeros(M, N, dtype=tdt(dtype), device="cuda")
     m.linear(a_d, w_d, b_d, 0, out)
-    assert rel_l2(host(out), acc) <= (4e-3 if dtype == "bf16" else 1e-6)
-    assert max_abs(host(out), acc) <= (3e-2 if dtype == "bf16" else 1e-4)
+    assert rel_l2(host(out), acc) <= (4e-3 if dtype in LOW else 1e-6)
+    assert max_abs(host(out), acc) <= (3e-2 if dtype in LOW else 1e-4)
     # bias + residual (fp32 read-modify-write)
     res = rng.standard_normal((M, N)).astype(np.float32)
     out = dev(res)
@@ -95,11 +104,11 @@ def test_linear_all_epilogues(dtype, M, N, K):
     out = torch.zeros(M, N, dtype=adt(dtype), device="cuda")
     m.linear(a_d, w_d, b_d, 2, out)
     want = orc.gelu(acc)
-    assert rel_l2(host(out), want) <= (4e-3 if dtype == "bf16" else 1e-6)
-    assert max_abs(host(out), want) <= (3e-2 if dtype == "bf16" else 1e-4)
+    assert rel_l2(host(out), want) <= (4e-3 if dtype in LOW else 1e-6)
+    assert max_abs(host(out), want) <= (3e-2 if dtype in LOW else 1e-4)
 
 
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "bf16b"])
 def test_linear_strided_input_and_row_guard(dtype):
     """a is a column slice of a wider matrix (lda > K); rows >= M of `out` stay untouched."""
     cfg, blocks, m = model_for(dtype, 256, 4, 1024, 68, 2)
@@ -112,7 +121,7 @@ def test_linear_strided_input_and_row_guard(dtype):
     out = torch.full((M + 60, N), 5.0, dtype=tdt(dtype), device="cuda")
     m.linear(wide_d[:, K:2 * K], dev(w, adt(dtype)), dev(bias), 0, out, M=M, lda=3 * K)
     want = orc.linear(quant_a(wide[:, K:2 * K], dtype), quant_a(w, dtype), bias.astype(np.float64))
-    assert rel_l2(host(out[:M]), want) <= (4e-3 if dtype == "bf16" else 1e-6)
+    assert rel_l2(host(out[:M]), want) <= (4e-3 if dtype in LOW else 1e-6)
     assert (host(out[M:]) == 5.0).all()
 
 
@@ -159,7 +168,7 @@ def test_scatter_rows_and_build_active():
 
 
 # ------------------------------------------------------------------ K3 attention (+ scores)
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "bf16b"])
 @pytest.mark.parametrize("S", [68, 320])
 @pytest.mark.parametrize("dh,H", [(64, 4), (80, 2)])
 @pytest.mark.parametrize("n,nG", [(1, 1), (2, 0), (12, 7), (41, 25), (77, 77)])
@@ -192,10 +201,10 @@ def test_attention_and_score_partials(dtype, S, dh, H, n, nG):
             want_o[b * n:(b + 1) * n, c] = z
             want_p[b, h] = p[flags[b].astype(bool)].sum(axis=0)
     got_o, got_p = host(o), host(partial)
-    assert rel_l2(got_o, want_o) <= (8e-3 if dtype == "bf16" else 1e-5)
-    assert max_abs(got_o, want_o) <= (3e-2 if dtype == "bf16" else 1e-4)
-    assert max_abs(got_p, want_p) <= (2e-2 if dtype == "bf16" else 1e-5) * max(1, nG) / 8 + 1e-6
-    assert np.allclose(got_p.sum(-1), nG, rtol=(5e-3 if dtype == "bf16" else 1e-5), atol=1e-6)   # each row sums to 1
+    assert rel_l2(got_o, want_o) <= (8e-3 if dtype in LOW else 1e-5)
+    assert max_abs(got_o, want_o) <= (3e-2 if dtype in LOW else 1e-4)
+    assert max_abs(got_p, want_p) <= (2e-2 if dtype in LOW else 1e-5) * max(1, nG) / 8 + 1e-6
+    assert np.allclose(got_p.sum(-1), nG, rtol=(5e-3 if dtype in LOW else 1e-5), atol=1e-6)   # each row sums to 1
     # scores off: partial buffer untouched
     partial2 = torch.full((B, H, S), -1.0, device="cuda")
     m.attention(q_d, 3 * D, n, dev(cache, tdt(dtype)), None, partial2, o)
@@ -241,7 +250,7 @@ def test_two_segment_attention_equals_scatter_then_attend(S, dh, H, n, nG):
     assert np.allclose(host(p_a).sum(-1), nG, rtol=5e-3, atol=1e-6)
 
 
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "bf16b"])
 def test_attention_uniform_and_peaked(dtype):
     S, B, H, dh, n = 68, 2, 4, 64, 5
     D = H * dh
@@ -255,8 +264,8 @@ def test_attention_uniform_and_peaked(dtype):
     m.attention(torch.zeros(B * n, D, dtype=tdt(dtype), device="cuda"), D, n, dev(cache, tdt(dtype)), dev(flags),
                 partial, o)
     vm = quant(cache, dtype)[1].mean(axis=1)
-    assert max_abs(host(o).reshape(B, n, D), np.repeat(vm[:, None], n, 1)) <= (4e-3 if dtype == "bf16" else 1e-5)
-    assert np.allclose(host(partial), n / S, rtol=1e-3 if dtype == "bf16" else 1e-5)
+    assert max_abs(host(o).reshape(B, n, D), np.repeat(vm[:, None], n, 1)) <= (4e-3 if dtype in LOW else 1e-5)
+    assert np.allclose(host(partial), n / S, rtol=1e-3 if dtype in LOW else 1e-5)
     # q = 64 * k_t -> one-hot on key t: o = V[t]; no inf/nan
     tsel = rng.integers(0, S, size=(B, n))
     kq = quant(cache, dtype)
@@ -265,7 +274,7 @@ def test_attention_uniform_and_peaked(dtype):
     got = host(o).reshape(B, n, D)
     assert np.isfinite(got).all()
     for b in range(B):
-        assert max_abs(got[b], kq[1, b, tsel[b]]) <= (2e-2 if dtype == "bf16" else 1e-4)
+        assert max_abs(got[b], kq[1, b, tsel[b]]) <= (2e-2 if dtype in LOW else 1e-4)
     assert np.allclose(host(partial).sum(-1), n, rtol=1e-3)
 
 

@@ -23,7 +23,11 @@ CASES = {
     "marb_slice": synth.CONFIGS["mar_b"].replace(L=3, E=1, B=4, T=6),
     # head_dim 80 (MAR-H-shaped rows)
     "marh_slice": synth.CONFIGS["mar_h"].replace(L=2, E=0, B=2, T=4),
+    # the same 16-bit stacks with bf16 projection operands (MARCHE_BF16) instead of fp16 ones
+    "tiny_bf16_bf16op": synth.CONFIGS["tiny"].replace(dtype="bf16"),
+    "marb_slice_bf16op": synth.CONFIGS["mar_b"].replace(L=3, E=1, B=4, T=6),
 }
+OPERAND = {name: ("bf16" if name.endswith("_bf16op") else "f16") for name in CASES}
 
 
 def oracle_run(cfg, blocks, hidden0, ratio, mode="marche"):
@@ -34,8 +38,8 @@ def oracle_run(cfg, blocks, hidden0, ratio, mode="marche"):
     return sets, log, cache
 
 
-def gpu_generation(cfg, blocks, sets, ratio):
-    m = make_model(cfg, blocks)
+def gpu_generation(cfg, blocks, sets, ratio, operand="f16"):
+    m = make_model(cfg, blocks, operand=operand)
     rows = [dev(synth.replacement_rows(cfg, t, sets[t].shape[1])) for t in range(cfg.T)]
     return m, Generation(m, sets, ratio, rows)
 
@@ -49,7 +53,7 @@ def test_teacher_forced_generation(case, ratio):
     blocks = synth.make_weights(cfg)
     hidden0 = synth.make_hidden(cfg)
     sets, log, cache = oracle_run(cfg, blocks, hidden0, ratio)
-    m, gen = gpu_generation(cfg, blocks, sets, ratio)
+    m, gen = gpu_generation(cfg, blocks, sets, ratio, OPERAND[case])
     forced = [idx_dev(rec["refresh"]) for rec in log]
     glog = gen.run(dev(hidden0), record=True, forced_refresh=forced)
     assert m.device_status() == 0
