@@ -38,10 +38,47 @@ import synth
 # MEASURED_PEAKS.json is absent.
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM traffic per launch of the dominant kernel classes from the committed ncu captures
-# (profiles/), bytes; None where no capture exists.
-NCU_TRAFFIC = {"gemm": 31.3e6,        # profiles/gemm_tcgen05_2cta_mar_l_rows4352.md (mean of the block's four GEMMs)
-               "attention": 183.6e6}  # profiles/attention_mma_mar_l_nA34.md
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_dram_traffic.txt")
+
+
+def load_ncu_traffic():
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel
+    classes, as written from an ncu capture by `bench.py --write-traffic <ncu raw csv>`:
+    lines `class bytes_per_launch launches`.  {} when the file is absent."""
+    out = {}
+    if os.path.exists(TRAFFIC_FILE):
+        for ln in open(TRAFFIC_FILE):
+            f = ln.split()
+            if len(f) >= 2 and not ln.startswith("#"):
+                out[f[0]] = float(f[1])
+    return out
+
+
+def write_ncu_traffic(csv_path):
+    """Reads `ncu -i <report> --page raw --csv` output and writes the mean DRAM bytes per launch of the
+    GEMM and attention kernels to profiles/ncu_dram_traffic.txt."""
+    import csv
+    rows = list(csv.reader(open(csv_path)))
+    hdr = next(r for r in rows if "Kernel Name" in r)
+    units = rows[rows.index(hdr) + 1]
+    i_name = hdr.index("Kernel Name")
+    i_rd, i_wr = hdr.index("dram__bytes_read.sum"), hdr.index("dram__bytes_write.sum")
+    scale = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
+    acc = {}
+    for r in rows[rows.index(hdr) + 2:]:
+        if len(r) <= max(i_rd, i_wr):
+            continue
+        cls = "gemm" if "gemm_tcgen05" in r[i_name] else ("attention" if "attention" in r[i_name] else None)
+        if cls is None:
+            continue
+        b = float(r[i_rd].replace(",", "")) * scale[units[i_rd]] + float(r[i_wr].replace(",", "")) * scale[units[i_wr]]
+        acc.setdefault(cls, []).append(b)
+    with open(TRAFFIC_FILE, "w") as f:
+        f.write("# mean dram__bytes_read.sum + dram__bytes_write.sum per launch, from %s\n" % os.path.basename(csv_path))
+        f.write("# class bytes_per_launch launches\n")
+        for cls, v in sorted(acc.items()):
+            f.write("%s %.0f %d\n" % (cls, float(np.mean(v)), len(v)))
+    print(open(TRAFFIC_FILE).read())
 
 
 def load_peaks():
@@ -282,7 +319,7 @@ def run_ours(args, cfg):
 
     ratio = args.ratio
     blocks = synth.make_weights(cfg)
-    m = Marche.from_config(cfg, upload_weights(blocks, cfg.dtype))
+    m = Marche.from_config(cfg, upload_weights(blocks, cfg.dtype, operand=args.operand))
     del blocks
     hidden0_np = synth.make_hidden(cfg)
     sets = synth.new_token_sets(cfg, synth.generation_orders(cfg))
@@ -324,7 +361,9 @@ def run_ours(args, cfg):
 
     line = {"metric": METRIC, "value": value, "unit": "images/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_gen, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "fp16 projections + bf16 attention/cache, fp32 accumulate" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+            "vs_baseline": None,
+            "dtype": ("%s projections + bf16 attention/cache, fp32 accumulate" % ("fp16" if args.operand == "f16" else "bf16"))
+                     if cfg.dtype == "bf16" else "f32", "data": "synthetic",
             "config": workload_config(cfg, ratio), "clocks": clock_info, "gpu_launches": int(launches),
             "ms_per_decoding_step": ms_gen / cfg.T}
 
@@ -350,9 +389,52 @@ def run_ours(args, cfg):
         dom = kernels[0]
         key = "gemm" if dom["bound"] == "tensor" else dom["kernel"]
         line["roofline"] = {"kernel": dom["kernel"], "bound": dom["bound"], "achieved": dom["achieved"], "peak": dom["peak"],
-                            "unit": dom["unit"], "frac": dom["frac"], "traffic": NCU_TRAFFIC.get(key),
+                            "unit": dom["unit"], "frac": dom["frac"], "traffic": load_ncu_traffic().get(key),
                             "peak_source": "%s (%s)" % (peak_kind, "sustained bf16 GEMM" if dom["bound"] == "tensor" else "device copy"),
                             "timing": "CUDA events in front of every launch, cache-aware steps of one generation of the timed workload"}
+
+        # ---- cost of each kernel class inside the REAL chain (launch overlap on, no events between
+        # kernels): the timed generation minus the same generation with that class left out.
+        if n_dec is None:
+            in_chain = {}
+            names = ("gather_layernorm", "gemm_qkv", "attention", "gemm_out_proj", "gemm_fc1_gelu", "gemm_fc2")
+            ms_ref = timed(lambda: gen.run(hidden0), 2)
+            for cls in names:
+                m.debug_skip_classes([cls])
+                gen.run(hidden0)
+                in_chain[cls] = ms_ref - timed(lambda: gen.run(hidden0), 2)
+            m.debug_skip_classes(names)
+            gen.run(hidden0)
+            ms_rest = timed(lambda: gen.run(hidden0), 2)
+            m.debug_skip_classes(())
+            gen.run(hidden0)                                   # leaves the buffers of a real generation behind
+            m.clear_device_status()
+            w_all = algorithmic_work(cfg, sched)
+            tot = sum(w_all["gemm_split"].values())
+            rows_ic = []
+            for cls in names:
+                ms = in_chain[cls]
+                if cls.startswith("gemm"):
+                    amount, peak, unit = w_all["gemm_flops"] * w_all["gemm_split"][cls] / tot / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s"
+                elif cls == "attention":
+                    amount, peak, unit = w_all["attention_bytes"] / 1e9, peaks["hbm_gbs"], "GB/s"
+                else:
+                    amount, peak, unit = w_all["gather_layernorm_bytes"] / 1e9, peaks["hbm_gbs"], "GB/s"
+                ach = amount / (ms * 1e-3) if ms > 0 else None
+                rows_ic.append({"kernel": cls, "ms": ms, "share": ms / ms_ref, "achieved": ach, "unit": unit, "peak": peak,
+                                "frac": None if ach is None else ach / peak})
+            gemm_ms = sum(in_chain[c] for c in names if c.startswith("gemm"))
+            line["kernels_in_chain"] = {
+                "method": "whole generation (all %d steps) timed as in the headline, minus the same generation with the "
+                          "class's launches left out; launch overlap stays on" % cfg.T,
+                "ms_per_step": ms_ref, "rows": rows_ic, "everything_else_ms": ms_rest,
+                "sum_ms": sum(in_chain.values()) + ms_rest,
+                "gemm_all": {"ms": gemm_ms, "achieved": w_all["gemm_flops"] / 1e12 / (gemm_ms * 1e-3), "unit": "TFLOP/s",
+                             "frac": w_all["gemm_flops"] / 1e12 / (gemm_ms * 1e-3) / peaks["bf16_tflops_sustained"]}}
+
+            if dom["bound"] == "tensor":
+                line["roofline"]["frac_in_chain"] = line["kernels_in_chain"]["gemm_all"]["frac"]
+                line["roofline"]["achieved_in_chain"] = line["kernels_in_chain"]["gemm_all"]["achieved"]
 
         # ---- the same generation captured once in a CUDA graph and replayed (no host launch cost at all)
         if n_dec is None:
@@ -381,7 +463,7 @@ def run_ours(args, cfg):
 
         # ---- each kernel on its own at the median cache-aware shape (no dependency gaps)
         n_mid = int(np.median([s_[1] for s_ in sched[1:]]))
-        line["kernels_isolated"] = {"n_active": n_mid, "rows": isolated_kernels(m, cfg, peaks, n_mid)}
+        line["kernels_isolated"] = {"n_active": n_mid, "rows": isolated_kernels(m, cfg, peaks, n_mid, args.operand)}
 
         # ---- this build's own full-recompute path (full step at every decoding step)
         gen.run(hidden0, mode="full")
@@ -404,7 +486,7 @@ def run_ours(args, cfg):
         # every step; decoder under the same schedule.  This is the shape the paper's own numbers are for.
         if 1 <= cfg.E < cfg.L and cfg.score_layer < cfg.L - 1:
             from paper_2506_12035_b200.binding import upload_mar_weights
-            m.set_mar_weights(upload_mar_weights(synth.make_mar_weights(cfg), cfg.dtype))
+            m.set_mar_weights(upload_mar_weights(synth.make_mar_weights(cfg), cfg.dtype, operand=args.operand))
             known = synth.known_token_sets(cfg, sets)
             gen.run_mar(hidden0, known)
             ms_ts = timed(lambda: gen.run_mar(hidden0, known), 2)
@@ -437,7 +519,7 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
-def isolated_kernels(m, cfg, peaks, n_active):
+def isolated_kernels(m, cfg, peaks, n_active, operand="f16"):
     """Each hot-path kernel timed on its own at one mid-run shape (n_active rows per sample):
     back-to-back launches through the single-kernel C calls (replayed from a CUDA graph), CUDA events around the batch, buffers
     rotated so that streamed operands come from HBM.  Unlike the per-class table of the generation,
@@ -446,7 +528,7 @@ def isolated_kernels(m, cfg, peaks, n_active):
     B, S, D, F, H = cfg.B, cfg.S, cfg.D, cfg.F, cfg.H
     M = B * n_active
     dev = "cuda"
-    act = torch.float16 if cfg.dtype == "bf16" else torch.float32
+    act = (torch.float16 if operand == "f16" else torch.bfloat16) if cfg.dtype == "bf16" else torch.float32
     typ = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
     eb = 2 if cfg.dtype == "bf16" else 4
     rot = 3
@@ -582,6 +664,21 @@ def run_microbench(args):
                           "us": us, "GB/s": nbytes / us * 1e-3, "frac_of_hbm": nbytes / us * 1e-3 / peaks["hbm_gbs"]}), flush=True)
 
 
+def spawn_replicas(n: int) -> int:
+    """`python bench.py --gpus N` without a launcher: starts one replica process per GPU with the
+    environment a launcher would have set (rank 0's JSON line goes to this process's stdout)."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env))
+    return max(p.wait() for p in procs)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -599,7 +696,15 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--microbench", action="store_true",
                     help="Appendix-B style attention micro-benchmark instead of the generation benchmark")
+    ap.add_argument("--operand", default="f16", choices=["f16", "bf16"],
+                    help="16-bit configs: element type of the projections' operands (f16 meets the 3e-2 bound at full depth)")
+    ap.add_argument("--write-traffic", default="", help="ncu raw csv -> profiles/ncu_dram_traffic.txt, then exit")
     args = ap.parse_args()
+    if args.write_traffic:
+        write_ncu_traffic(args.write_traffic)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.microbench:
+        sys.exit(spawn_replicas(args.gpus))
     cfg = synth.CONFIGS[args.config]
     if args.blocks:
         cfg = cfg.replace(L=args.blocks, E=min(cfg.E, max(0, args.blocks - 2)))

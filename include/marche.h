@@ -492,6 +492,13 @@ unsigned long long marche_launch_count(const marche_ctx* ctx);
 int marche_profile_begin(marche_ctx* ctx);
 int marche_profile_end(marche_ctx* ctx, marche_stream stream, float* ms_per_class, int* launches_per_class);
 const char* marche_kernel_class_name(int kernel_class);
+/* Measurement hook for the cost of a kernel class INSIDE the real launch chain (launch overlap on, no
+ * events between kernels): while bit c of `class_mask` is set, the step calls do not launch the kernels
+ * of class c, so (time of a step) - (time of the same step with the class left out) is what that
+ * class costs in the chain.  The results of such a step are garbage (stale buffers are read) but every
+ * index stays in range.  Only MARCHE_KC_GATHER_LN, _GEMM_QKV, _ATTENTION, _GEMM_O, _GEMM_FC1 and
+ * _GEMM_FC2 may be left out (MARCHE_EINVAL otherwise); 0 restores the normal step. */
+int marche_debug_skip_classes(marche_ctx* ctx, unsigned class_mask);
 void marche_clear_device_status(marche_ctx* ctx);
 
 #ifdef __cplusplus

@@ -97,6 +97,7 @@ _SIGNATURES = {
     "marche_set_tuning": (C.c_int, [_vp, C.POINTER(MarcheTuning)]),
     "marche_check_status": (C.c_int, [_vp, _vp]),
     "marche_debug_bounded_wait": (C.c_int, [_vp, C.c_longlong, _vp]),
+    "marche_debug_skip_classes": (C.c_int, [_vp, C.c_uint]),
 }
 EXPORTED_SYMBOLS = tuple(_SIGNATURES)
 
@@ -418,6 +419,16 @@ class Marche:
 
     def debug_bounded_wait(self, limit_cycles: int, stream=None):
         self._check(self.lib.marche_debug_bounded_wait(self.h, limit_cycles, _stream(stream)))
+
+    KERNEL_CLASSES = ("step_flags", "gather_layernorm", "gemm_qkv", "scatter_kv", "attention", "gemm_out_proj",
+                      "gemm_fc1_gelu", "gemm_fc2", "scatter_rows", "topk", "other")
+
+    def debug_skip_classes(self, names: Sequence[str] = ()):
+        """Measurement hook: the named kernel classes are not launched until called again with ()."""
+        mask = 0
+        for n in names:
+            mask |= 1 << self.KERNEL_CLASSES.index(n)
+        self._check(self.lib.marche_debug_skip_classes(self.h, mask))
 
     def device_status(self) -> int:
         return self.lib.marche_device_status(self.h)

@@ -38,6 +38,7 @@ struct marche_ctx {
   int score_layer = 0;
   std::vector<int> extra_score_layers;                // blocks that also accumulate scores (analysis only)
   marche_tuning tune;                                 // kernel-selection switches (marche_set_tuning)
+  unsigned skip_mask = 0;                             // measurement hook: kernel classes that are not launched
   std::vector<std::pair<const void*, bool>> caches;  // (cache pointer, filled)
   int* status_host = nullptr;                         // pinned, mapped
   int* status_dev = nullptr;
@@ -154,6 +155,8 @@ GemmTuning gemm_tuning(const marche_ctx* ctx) {
   return g;
 }
 
+inline bool skipped(const marche_ctx* ctx, int cls) { return (ctx->skip_mask >> cls) & 1u; }
+
 int refresh_count(float ratio, int S, int n_cand) {
   const int want = (int)std::floor((double)ratio * (double)S + 0.5);
   return want < n_cand ? (want < 0 ? 0 : want) : n_cand;
@@ -180,6 +183,7 @@ bool qkv_scatter_fused(const marche_ctx* ctx, int M, int S) {
 
 int do_linear(marche_ctx* ctx, int cls, const void* a, int lda, int M, const void* w, const float* bias, int N, int K,
               int epi, void* out, cudaStream_t st, int* turn = nullptr, const KvScatter* kv = nullptr) {
+  if (skipped(ctx, cls)) return MARCHE_OK;
   if (!ctx->bf16) {
     if (M > 0) mark(ctx, cls, st);
     MARCHE_TRY(launch_gemm_simt((const float*)a, lda, M, (const float*)w, bias, N, K, epi, (float*)out, st), "gemm");
@@ -202,6 +206,7 @@ int do_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void* ca
                  float* partial, void* o, cudaStream_t st, int S_kv = 0) {
   const marche_config& c = ctx->cfg;
   const int S = S_kv > 0 ? S_kv : c.seq_len;            // tokens per sample in cache_layer [2][B][S][D]
+  if (skipped(ctx, MARCHE_KC_ATTENTION)) return MARCHE_OK;
   if (!ctx->bf16) {
     if (n > 0) mark(ctx, MARCHE_KC_ATTENTION, st);
     MARCHE_TRY(launch_attention_simt((const float*)q, ld_q, c.batch, n, S, c.n_heads, c.head_dim, (const float*)cache_layer,
@@ -273,8 +278,10 @@ int run_blocks(marche_ctx* ctx, int l_begin, int l_end, const float* gather_src,
     const int slot = is_new ? score_slot(ctx, l) : -1;
     const uint8_t* flags_l = slot >= 0 ? is_new : nullptr;
     float* partial_l = bf.partial + (size_t)(slot > 0 ? slot : 0) * B * c.n_heads * c.seq_len;
-    mark(ctx, MARCHE_KC_GATHER_LN, st);
-    if (l == l_begin && gather_src)
+    const bool skip_ln = skipped(ctx, MARCHE_KC_GATHER_LN);
+    if (!skip_ln) mark(ctx, MARCHE_KC_GATHER_LN, st);
+    if (skip_ln) {
+    } else if (l == l_begin && gather_src)
       MARCHE_TRY(launch_gather_layernorm(ctx->a_kind, gather_src, src_rows, idx, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
                                          x, bf.u, st), "gather_layernorm");
     else
@@ -305,9 +312,11 @@ int run_blocks(marche_ctx* ctx, int l_begin, int l_end, const float* gather_src,
     }
     rc = do_linear(ctx, MARCHE_KC_GEMM_O, bf.o, D, M, bw.w_o, bw.b_o, D, D, MARCHE_EPI_BIAS_RESIDUAL, x, st, bf.turn);
     if (rc) return rc;
-    mark(ctx, MARCHE_KC_GATHER_LN, st);
-    MARCHE_TRY(launch_gather_layernorm(ctx->a_kind, x, nA, nullptr, B, nA, D, bw.ln2_g, bw.ln2_b, ctx->eps, nullptr,
-                                       bf.u, st), "layernorm2");
+    if (!skip_ln) {
+      mark(ctx, MARCHE_KC_GATHER_LN, st);
+      MARCHE_TRY(launch_gather_layernorm(ctx->a_kind, x, nA, nullptr, B, nA, D, bw.ln2_g, bw.ln2_b, ctx->eps, nullptr,
+                                         bf.u, st), "layernorm2");
+    }
     rc = do_linear(ctx, MARCHE_KC_GEMM_FC1, bf.u, D, M, bw.w_fc1, bw.b_fc1, F, D, MARCHE_EPI_BIAS_GELU, bf.g, st);
     if (rc) return rc;
     rc = do_linear(ctx, MARCHE_KC_GEMM_FC2, bf.g, F, M, bw.w_fc2, bw.b_fc2, D, F, MARCHE_EPI_BIAS_RESIDUAL, x, st, bf.turn);
@@ -955,6 +964,15 @@ int marche_set_tuning(marche_ctx* ctx, const marche_tuning* t) {
   if (t->attention_tc_min_rows < 0) return MARCHE_EINVAL;
   ctx->tune = *t;
   pdl_switch() = t->pdl != 0;
+  return MARCHE_OK;
+}
+
+int marche_debug_skip_classes(marche_ctx* ctx, unsigned class_mask) {
+  if (!ctx) return MARCHE_EINVAL;
+  const unsigned allowed = (1u << MARCHE_KC_GATHER_LN) | (1u << MARCHE_KC_GEMM_QKV) | (1u << MARCHE_KC_ATTENTION) |
+                           (1u << MARCHE_KC_GEMM_O) | (1u << MARCHE_KC_GEMM_FC1) | (1u << MARCHE_KC_GEMM_FC2);
+  if (class_mask & ~allowed) return MARCHE_EINVAL;
+  ctx->skip_mask = class_mask;
   return MARCHE_OK;
 }
 

@@ -39,3 +39,21 @@ def test_single_process_passthrough():
     import bench
     assert bench.max_over_ranks(12.5, device="cpu") == 12.5
     assert bench.aggregate_images_per_s(64, 500.0, 1) == 128.0
+
+
+def test_bench_starts_its_own_replicas_when_no_launcher_did():
+    """`python bench.py --gpus 2` with no WORLD_SIZE in the environment starts two rank processes itself
+    (checked on the reference arm, which needs no GPU: rank 0 alone works and prints, rank 1 exits 0)."""
+    import json
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--impl", "reference", "--config", "tiny",
+                        "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["value"] > 0
