@@ -446,13 +446,14 @@ int marche_attention_two_segment(marche_ctx* ctx, const void* qkv, int ld, int n
  * are the measured winners on B200; the alternatives exist for measurements and for the tests that
  * pin them to the same results.  None of them changes what is computed, only which kernel does it;
  * `pdl` is process-wide (it is a property of how kernels are launched). */
-enum { MARCHE_ATTENTION_AUTO = 0, MARCHE_ATTENTION_MMA = 1, MARCHE_ATTENTION_TCGEN05 = 2 };
+enum { MARCHE_ATTENTION_AUTO = 0, MARCHE_ATTENTION_MMA = 1, MARCHE_ATTENTION_TCGEN05 = 2,
+       MARCHE_ATTENTION_TCGEN05_TWO_PASS = 3 /* the two-pass tcgen05 kernel also where no scores are taken */ };
 enum { MARCHE_GEMM_AUTO = 0, MARCHE_GEMM_SINGLE = 1, MARCHE_GEMM_PAIR = 2 };
 typedef struct {
   int32_t stream_k;              /* 1: fc2-sized residual projections use stream-K with ordered reduce-adds   */
   int32_t fuse_qkv_scatter;      /* 1: the QKV projection's epilogue writes K, V into the cache (no K5 launch)*/
   int32_t attention_kernel;      /* MARCHE_ATTENTION_*: AUTO picks by active rows and head_dim                 */
-  int32_t attention_tc_min_rows; /* AUTO: tcgen05 attention above this many active rows (head_dim 64)          */
+  int32_t attention_tc_min_rows; /* AUTO: tcgen05 attention above this many active rows (head_dim 64; 60)      */
   int32_t two_segment_attention; /* 1: the step uses marche_attention_two_segment instead of K5 + K3           */
   int32_t gemm_kernel;           /* MARCHE_GEMM_*: AUTO = CTA-pair kernel above 128 rows                       */
   int32_t tail_split;            /* 0 off, 1 cost model, 2 / 4 forced: column slices in a partial last round   */
@@ -499,6 +500,12 @@ const char* marche_kernel_class_name(int kernel_class);
  * index stays in range.  Only MARCHE_KC_GATHER_LN, _GEMM_QKV, _ATTENTION, _GEMM_O, _GEMM_FC1 and
  * _GEMM_FC2 may be left out (MARCHE_EINVAL otherwise); 0 restores the normal step. */
 int marche_debug_skip_classes(marche_ctx* ctx, unsigned class_mask);
+/* The complementary hook: while bit c is set, every launch of class c is issued twice in a row (same
+ * arguments).  (time with the class doubled) - (time of the normal step) is the class's cost in the real
+ * chain under the clocks and power the real chain runs at, which leaving a class out does not preserve
+ * on a power-capped GPU.  Doubling is harmless for the values except that the two residual projections
+ * add their result twice; use it for timing only.  Same classes, same errors. */
+int marche_debug_repeat_classes(marche_ctx* ctx, unsigned class_mask);
 void marche_clear_device_status(marche_ctx* ctx);
 
 #ifdef __cplusplus

@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmarche.so")
 
 MARCHE_F32, MARCHE_BF16, MARCHE_BF16_F16OP = 0, 1, 2
-ATTENTION_AUTO, ATTENTION_MMA, ATTENTION_TCGEN05 = 0, 1, 2
+ATTENTION_AUTO, ATTENTION_MMA, ATTENTION_TCGEN05, ATTENTION_TCGEN05_TWO_PASS = 0, 1, 2, 3
 GEMM_AUTO, GEMM_SINGLE, GEMM_PAIR = 0, 1, 2
 EPI_BIAS, EPI_BIAS_RESIDUAL, EPI_BIAS_GELU = 0, 1, 2
 ERRORS = {-1: "EINVAL", -2: "ESHAPE", -3: "EWORKSPACE", -4: "ECACHE", -5: "EINDEX", -6: "ECUDA", -7: "ETIMEOUT"}
@@ -98,6 +98,7 @@ _SIGNATURES = {
     "marche_check_status": (C.c_int, [_vp, _vp]),
     "marche_debug_bounded_wait": (C.c_int, [_vp, C.c_longlong, _vp]),
     "marche_debug_skip_classes": (C.c_int, [_vp, C.c_uint]),
+    "marche_debug_repeat_classes": (C.c_int, [_vp, C.c_uint]),
 }
 EXPORTED_SYMBOLS = tuple(_SIGNATURES)
 
@@ -429,6 +430,13 @@ class Marche:
         for n in names:
             mask |= 1 << self.KERNEL_CLASSES.index(n)
         self._check(self.lib.marche_debug_skip_classes(self.h, mask))
+
+    def debug_repeat_classes(self, names: Sequence[str] = ()):
+        """Measurement hook: every launch of the named kernel classes is issued twice until called again with ()."""
+        mask = 0
+        for n in names:
+            mask |= 1 << self.KERNEL_CLASSES.index(n)
+        self._check(self.lib.marche_debug_repeat_classes(self.h, mask))
 
     def device_status(self) -> int:
         return self.lib.marche_device_status(self.h)

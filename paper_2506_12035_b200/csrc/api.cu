@@ -39,6 +39,7 @@ struct marche_ctx {
   std::vector<int> extra_score_layers;                // blocks that also accumulate scores (analysis only)
   marche_tuning tune;                                 // kernel-selection switches (marche_set_tuning)
   unsigned skip_mask = 0;                             // measurement hook: kernel classes that are not launched
+  unsigned repeat_mask = 0;                           // measurement hook: kernel classes that are launched twice
   std::vector<std::pair<const void*, bool>> caches;  // (cache pointer, filled)
   int* status_host = nullptr;                         // pinned, mapped
   int* status_dev = nullptr;
@@ -111,7 +112,7 @@ marche_tuning default_tuning() {
   t.stream_k = 1;
   t.fuse_qkv_scatter = 1;
   t.attention_kernel = MARCHE_ATTENTION_AUTO;
-  t.attention_tc_min_rows = 96;
+  t.attention_tc_min_rows = 60;
   t.two_segment_attention = 0;
   t.gemm_kernel = MARCHE_GEMM_AUTO;
   t.tail_split = 1;
@@ -156,6 +157,7 @@ GemmTuning gemm_tuning(const marche_ctx* ctx) {
 }
 
 inline bool skipped(const marche_ctx* ctx, int cls) { return (ctx->skip_mask >> cls) & 1u; }
+inline int launches_of(const marche_ctx* ctx, int cls) { return ((ctx->repeat_mask >> cls) & 1u) ? 2 : 1; }
 
 int refresh_count(float ratio, int S, int n_cand) {
   const int want = (int)std::floor((double)ratio * (double)S + 0.5);
@@ -192,13 +194,15 @@ int do_linear(marche_ctx* ctx, int cls, const void* a, int lda, int M, const voi
   // 16-bit contexts run on the tensor cores or not at all
   if (N % 128 || K % 64) return MARCHE_ESHAPE;
   if (lda % 8 || (((uintptr_t)a | (uintptr_t)w | (uintptr_t)out) & 15)) return misaligned(ctx, "projection");
-  if (M > 0) mark(ctx, cls, st);
   const bool pair = ctx->tune.gemm_kernel == MARCHE_GEMM_PAIR || (ctx->tune.gemm_kernel == MARCHE_GEMM_AUTO && M > 128);
-  if (pair)
-    MARCHE_TRY(launch_gemm_tcgen05_2cta(a, lda, M, w, bias, N, K, epi, out, ctx->a_bf16, ctx->status_dev, st,
-                                        gemm_tuning(ctx), turn, kv), "gemm_tcgen05_2cta");
-  else
-    MARCHE_TRY(launch_gemm_tcgen05(a, lda, M, w, bias, N, K, epi, out, ctx->a_bf16, ctx->status_dev, st), "gemm_tcgen05");
+  for (int r = 0; r < launches_of(ctx, cls); ++r) {
+    if (M > 0) mark(ctx, cls, st);
+    if (pair)
+      MARCHE_TRY(launch_gemm_tcgen05_2cta(a, lda, M, w, bias, N, K, epi, out, ctx->a_bf16, ctx->status_dev, st,
+                                          gemm_tuning(ctx), turn, kv), "gemm_tcgen05_2cta");
+    else
+      MARCHE_TRY(launch_gemm_tcgen05(a, lda, M, w, bias, N, K, epi, out, ctx->a_bf16, ctx->status_dev, st), "gemm_tcgen05");
+  }
   return MARCHE_OK;
 }
 
@@ -214,22 +218,30 @@ int do_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void* ca
     return MARCHE_OK;
   }
   if (ld_q % 2 || ((uintptr_t)q & 3) || ((uintptr_t)cache_layer & 15) || ((uintptr_t)o & 15)) return misaligned(ctx, "attention");
+  for (int rep_i = 0; rep_i < launches_of(ctx, MARCHE_KC_ATTENTION); ++rep_i) {
   if (n > 0) mark(ctx, MARCHE_KC_ATTENTION, st);
-  // Two tensor-core kernels.  At small active sets the step is bound by streaming the cache and the
-  // mma.sync kernel (several small CTAs per SM, one pass) is faster: 41 us vs 69 us at n = 41.  Once
-  // the legacy tensor path saturates (about 250 TFLOP/s) the tcgen05 kernel wins: 109 vs 172 us at
-  // n = 122 (S 1088), 840 vs 1100 us at n = S = 1088, and earlier for the two-pass scoring flavour
-  // (97 vs 143 us at n = 77).  marche_tuning.attention_kernel forces one of them; head_dim 80 has only the former.
+  // Three tensor-core kernels.  At small active sets the step is bound by streaming the cache and the
+  // mma.sync kernel (several small CTAs per SM, one pass) is fastest: 43 us vs 51 us at n = 41 (S 320).
+  // From about 60 rows the single-pass tcgen05 kernel wins (S 320: 53 vs 58 us at n = 64, 54 vs 110 us at
+  // n = 77, 151 vs 303 us at n = 320; S 1088: 83 vs 252 us at n = 116, 137 vs 256 us at n = 159).  The
+  // relevance scores need final weights, hence the two-pass tcgen05 kernel there (74 vs 143 us at n = 77).
+  // marche_tuning.attention_kernel forces one of them; head_dim 80 has only the mma.sync kernel.
   const int tc_min = is_new ? 64 : ctx->tune.attention_tc_min_rows;
+  const int ak = ctx->tune.attention_kernel;
   const bool tc5 = c.head_dim == 64 && ld_q % 8 == 0 && ((uintptr_t)q & 15) == 0 &&
-                   (ctx->tune.attention_kernel == MARCHE_ATTENTION_TCGEN05 ||
-                    (ctx->tune.attention_kernel == MARCHE_ATTENTION_AUTO && n > tc_min));
-  if (tc5)
+                   (ak == MARCHE_ATTENTION_TCGEN05 || ak == MARCHE_ATTENTION_TCGEN05_TWO_PASS ||
+                    (ak == MARCHE_ATTENTION_AUTO && n > tc_min));
+  // plain flavour: single-pass streaming kernel; the relevance scores need final weights, i.e. two passes
+  if (tc5 && !is_new && ak != MARCHE_ATTENTION_TCGEN05_TWO_PASS)
+    MARCHE_TRY(launch_attention_tc_stream(q, ld_q, c.batch, n, S, c.n_heads, c.head_dim, cache_layer, o, ctx->a_bf16,
+                                          ctx->status_dev, st), "attention_tc_stream");
+  else if (tc5)
     MARCHE_TRY(launch_attention_tcgen05(q, ld_q, c.batch, n, S, c.n_heads, c.head_dim, cache_layer, is_new,
                                         partial, o, ctx->a_bf16, ctx->status_dev, st), "attention_tcgen05");
   else
     MARCHE_TRY(launch_attention_mma(q, ld_q, c.batch, n, S, c.n_heads, c.head_dim, cache_layer, is_new,
                                     partial, o, ctx->a_bf16, ctx->status_dev, st), "attention_mma");
+  }
   return MARCHE_OK;
 }
 
@@ -280,13 +292,15 @@ int run_blocks(marche_ctx* ctx, int l_begin, int l_end, const float* gather_src,
     float* partial_l = bf.partial + (size_t)(slot > 0 ? slot : 0) * B * c.n_heads * c.seq_len;
     const bool skip_ln = skipped(ctx, MARCHE_KC_GATHER_LN);
     if (!skip_ln) mark(ctx, MARCHE_KC_GATHER_LN, st);
-    if (skip_ln) {
-    } else if (l == l_begin && gather_src)
-      MARCHE_TRY(launch_gather_layernorm(ctx->a_kind, gather_src, src_rows, idx, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
-                                         x, bf.u, st), "gather_layernorm");
-    else
-      MARCHE_TRY(launch_gather_layernorm(ctx->a_kind, x, nA, nullptr, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
-                                         nullptr, bf.u, st), "layernorm1");
+    for (int r = 0; r < (skip_ln ? 0 : launches_of(ctx, MARCHE_KC_GATHER_LN)); ++r) {
+      if (r) mark(ctx, MARCHE_KC_GATHER_LN, st);
+      if (l == l_begin && gather_src)
+        MARCHE_TRY(launch_gather_layernorm(ctx->a_kind, gather_src, src_rows, idx, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
+                                           x, bf.u, st), "gather_layernorm");
+      else
+        MARCHE_TRY(launch_gather_layernorm(ctx->a_kind, x, nA, nullptr, B, nA, D, bw.ln1_g, bw.ln1_b, ctx->eps,
+                                           nullptr, bf.u, st), "layernorm1");
+    }
     const bool fused_kv = qkv_scatter_fused(ctx, M, S);
     const KvScatter kvs = {kv_idx, cache_l, nA, S, B, D};
     int rc = do_linear(ctx, MARCHE_KC_GEMM_QKV, bf.u, D, M, bw.w_qkv, bw.b_qkv, 3 * D, D, fused_kv ? 4 : MARCHE_EPI_BIAS,
@@ -312,7 +326,7 @@ int run_blocks(marche_ctx* ctx, int l_begin, int l_end, const float* gather_src,
     }
     rc = do_linear(ctx, MARCHE_KC_GEMM_O, bf.o, D, M, bw.w_o, bw.b_o, D, D, MARCHE_EPI_BIAS_RESIDUAL, x, st, bf.turn);
     if (rc) return rc;
-    if (!skip_ln) {
+    for (int r = 0; r < (skip_ln ? 0 : launches_of(ctx, MARCHE_KC_GATHER_LN)); ++r) {
       mark(ctx, MARCHE_KC_GATHER_LN, st);
       MARCHE_TRY(launch_gather_layernorm(ctx->a_kind, x, nA, nullptr, B, nA, D, bw.ln2_g, bw.ln2_b, ctx->eps, nullptr,
                                          bf.u, st), "layernorm2");
@@ -957,7 +971,7 @@ int marche_get_tuning(const marche_ctx* ctx, marche_tuning* out) {
 
 int marche_set_tuning(marche_ctx* ctx, const marche_tuning* t) {
   if (!ctx || !t) return MARCHE_EINVAL;
-  if (t->attention_kernel < MARCHE_ATTENTION_AUTO || t->attention_kernel > MARCHE_ATTENTION_TCGEN05) return MARCHE_EINVAL;
+  if (t->attention_kernel < MARCHE_ATTENTION_AUTO || t->attention_kernel > MARCHE_ATTENTION_TCGEN05_TWO_PASS) return MARCHE_EINVAL;
   if (t->gemm_kernel < MARCHE_GEMM_AUTO || t->gemm_kernel > MARCHE_GEMM_PAIR) return MARCHE_EINVAL;
   if (t->tail_split != 0 && t->tail_split != 1 && t->tail_split != 2 && t->tail_split != 4) return MARCHE_EINVAL;
   if (t->tile_n != 0 && t->tile_n != 128) return MARCHE_EINVAL;
@@ -967,12 +981,20 @@ int marche_set_tuning(marche_ctx* ctx, const marche_tuning* t) {
   return MARCHE_OK;
 }
 
+namespace {
+constexpr unsigned kHookClasses = (1u << MARCHE_KC_GATHER_LN) | (1u << MARCHE_KC_GEMM_QKV) | (1u << MARCHE_KC_ATTENTION) |
+                                  (1u << MARCHE_KC_GEMM_O) | (1u << MARCHE_KC_GEMM_FC1) | (1u << MARCHE_KC_GEMM_FC2);
+}
+
 int marche_debug_skip_classes(marche_ctx* ctx, unsigned class_mask) {
-  if (!ctx) return MARCHE_EINVAL;
-  const unsigned allowed = (1u << MARCHE_KC_GATHER_LN) | (1u << MARCHE_KC_GEMM_QKV) | (1u << MARCHE_KC_ATTENTION) |
-                           (1u << MARCHE_KC_GEMM_O) | (1u << MARCHE_KC_GEMM_FC1) | (1u << MARCHE_KC_GEMM_FC2);
-  if (class_mask & ~allowed) return MARCHE_EINVAL;
+  if (!ctx || (class_mask & ~kHookClasses)) return MARCHE_EINVAL;
   ctx->skip_mask = class_mask;
+  return MARCHE_OK;
+}
+
+int marche_debug_repeat_classes(marche_ctx* ctx, unsigned class_mask) {
+  if (!ctx || (class_mask & ~kHookClasses)) return MARCHE_EINVAL;
+  ctx->repeat_mask = class_mask;
   return MARCHE_OK;
 }
 

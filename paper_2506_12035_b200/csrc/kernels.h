@@ -109,6 +109,11 @@ cudaError_t launch_attention_tcgen05(const void* q, int ld_q, int B, int n, int 
                                      const void* cache_layer, const uint8_t* is_new, float* score_partial, void* o,
                                      bool o_bf16, int* status, cudaStream_t st);
 
+// K3 on tcgen05, single pass with online softmax, persistent over (sample, head) items, P kept in tensor
+// memory (head_dim 64, no relevance scores).  Same alignment rules as launch_attention_tcgen05, o 16-byte aligned.
+cudaError_t launch_attention_tc_stream(const void* q, int ld_q, int B, int n, int S, int H, int dh,
+                                       const void* cache_layer, void* o, bool o_bf16, int* status, cudaStream_t st);
+
 // K3, two-segment flavour (Eq. 6-10 without concatenation, then the cache write-back of Algorithm 1
 // line 11 by the same kernel): fresh K/V are columns k_off / v_off of the compact qkv buffer
 // [B*n][ld]; active_idx NULL = identity.  Same type and alignment rules as launch_attention_mma.

@@ -78,7 +78,7 @@ def test_tuning_alternatives_compute_the_same_step():
     blocks = synth.make_weights(cfg)
     m = make_model(cfg, blocks)
     defaults = m.get_tuning()
-    assert defaults == dict(stream_k=1, fuse_qkv_scatter=1, attention_kernel=0, attention_tc_min_rows=96,
+    assert defaults == dict(stream_k=1, fuse_qkv_scatter=1, attention_kernel=0, attention_tc_min_rows=60,
                             two_segment_attention=0, gemm_kernel=0, tail_split=1, tile_n=0, pdl=1)
     rng = np.random.default_rng(1)
     hidden_np = synth.make_hidden(cfg)
@@ -93,6 +93,7 @@ def test_tuning_alternatives_compute_the_same_step():
     hidden = dev(hidden_np)
     ma, rl = TOL["bf16"]
     variants = [dict(), dict(fuse_qkv_scatter=0), dict(two_segment_attention=1), dict(attention_kernel=binding.ATTENTION_TCGEN05),
+                dict(attention_kernel=binding.ATTENTION_TCGEN05_TWO_PASS),
                 dict(attention_kernel=binding.ATTENTION_MMA, attention_tc_min_rows=8), dict(gemm_kernel=binding.GEMM_SINGLE),
                 dict(gemm_kernel=binding.GEMM_PAIR, tile_n=128), dict(stream_k=0, tail_split=0), dict(tail_split=4), dict(pdl=0)]
     for v in variants:
@@ -105,7 +106,7 @@ def test_tuning_alternatives_compute_the_same_step():
         assert max_abs(host(cache[:, 0]), oc.K) <= ma and max_abs(host(cache[:, 1]), oc.V) <= ma, v
         assert np.array_equal(R.cpu().numpy(), orc.select_refresh(scores.cpu().numpy(), G, None, R.shape[1])), v
     m.set_tuning(**defaults)
-    for bad in (dict(attention_kernel=3), dict(gemm_kernel=-1), dict(tail_split=3), dict(tile_n=64)):
+    for bad in (dict(attention_kernel=4), dict(gemm_kernel=-1), dict(tail_split=3), dict(tile_n=64)):
         with pytest.raises(MarcheError) as e:
             m.set_tuning(**bad)
         assert e.value.code == -1

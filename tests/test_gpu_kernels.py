@@ -437,3 +437,49 @@ def test_attention_many_rows(S, dh, H, n, nG):
     m.attention(dev(q, tdt(dtype)), 3 * D, n, dev(cache, tdt(dtype)), None, None, o2)       # plain flavour
     assert rel_l2(host(o2), want_o) <= 8e-3 and max_abs(host(o2), want_o) <= 3e-2
     assert m.device_status() == 0
+
+
+@pytest.mark.parametrize("operand", ["bf16", "bf16b"])
+@pytest.mark.parametrize("B,H,S,n", [(2, 4, 68, 5), (2, 4, 128, 128), (3, 4, 320, 41), (40, 4, 320, 41), (2, 4, 320, 129),
+                                     (2, 4, 320, 320), (100, 4, 320, 77), (2, 16, 1088, 122), (2, 16, 1088, 159),
+                                     (1, 4, 1088, 1088), (2, 4, 2048, 300), (37, 8, 300, 257)])
+def test_attention_single_pass_tcgen05(operand, B, H, S, n):
+    """The single-pass tcgen05 kernel (weights kept in tensor memory, persistent over (sample, head) items) on
+    its own: one, two and more query tiles, one key tile up to sixteen with ragged tails, more items than SMs,
+    and logits whose row maximum keeps growing from tile to tile (the lazy rescaling of the accumulator)."""
+    from paper_2506_12035_b200 import binding
+    dh = 64
+    D = H * dh
+    if operand == "bf16b" and B * H * n * S > 3e6:
+        pytest.skip("one operand type is enough for the large shapes")
+    cfg, blocks, m = model_for(operand, D, H, 128, S, B)
+    m.set_tuning(attention_kernel=binding.ATTENTION_TCGEN05)
+    rng = np.random.default_rng(B + H + S + n)
+    cache = rng.standard_normal((2, B, S, D)).astype(np.float32)
+    # (i) ordinary logits; (ii) logits that grow with the key index: every tile raises the row maximum by
+    # far more than 2^8, so each tile rescales the accumulator; (iii) one-hot rows on a late key
+    q_rand = (rng.standard_normal((B * n, D)) * 3.0).astype(np.float32)
+    ramp = np.linspace(0.0, 40.0, S, dtype=np.float32)
+    cache_ramp = cache.copy()
+    cache_ramp[0, :, :, 0::dh] = ramp[None, :, None]                   # first channel of every head's keys
+    q_ramp = q_rand.copy()
+    q_ramp[:, 0::dh] = 16.0                                            # logit contribution 16 * ramp / 8 = 0 .. 80
+    kq = quant(cache, "bf16")
+    tsel = rng.integers(max(0, S - 40), S, size=(B, n))
+    q_hot = np.stack([kq[0, b, tsel[b]] for b in range(B)]).reshape(B * n, D).astype(np.float32) * 64.0
+    sample_b = sorted(set([0, B // 2, B - 1]))
+    for name, q, cch in (("random", q_rand, cache), ("ramp", q_ramp, cache_ramp), ("one-hot", q_hot, cache)):
+        o = torch.zeros(B * n, D, dtype=adt(operand), device="cuda")
+        m.attention(dev(q, torch.bfloat16), D, n, dev(cch, torch.bfloat16), None, None, o)
+        torch.cuda.synchronize()
+        assert m.device_status() == 0
+        got = host(o).reshape(B, n, D)
+        assert np.isfinite(got).all(), name
+        qq, cc = quant(q, "bf16").reshape(B, n, D), quant(cch, "bf16")
+        for b in sample_b:
+            want = np.zeros((n, D))
+            for h in range(H):
+                c = slice(h * dh, (h + 1) * dh)
+                want[:, c], _ = orc.softmax_attention(qq[b][:, c], cc[0, b][:, c], cc[1, b][:, c])
+            assert rel_l2(got[b], want) <= 8e-3 and max_abs(got[b], want) <= 3e-2, \
+                "%s b=%d: max-abs %.3g rel-L2 %.3g" % (name, b, max_abs(got[b], want), rel_l2(got[b], want))
