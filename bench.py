@@ -350,11 +350,27 @@ def run_ours(args, cfg):
     for _ in range(args.warmup):
         gen.run(hidden0, n_steps=n_dec)
     torch.cuda.synchronize()
+    # The timed step: the whole generation recorded once as a CUDA graph and replayed (the kernels, their
+    # arguments and their order are exactly those of the stream-launched generation; what goes away is the
+    # host's per-launch work).  --stream-launch, or a failed capture, times the stream-launched generation.
+    graph, per_replay, launch_mode = None, 0, "stream launches"
+    if not args.stream_launch and n_dec is None:
+        try:
+            l0 = m.launch_count()
+            graph = gen.capture(hidden0)
+            per_replay = (m.launch_count() - l0) // 2              # one eager generation, one recorded
+            for _ in range(2):
+                graph.replay()
+            torch.cuda.synchronize()
+            launch_mode = "one CUDA graph per generation (%d kernel nodes)" % per_replay
+        except Exception as exc:
+            graph, launch_mode = None, "stream launches (graph capture failed: %s)" % str(exc)[:120]
+    step_fn = (lambda: graph.replay()) if graph is not None else (lambda: gen.run(hidden0, n_steps=n_dec))
     clocks = ClockSampler(local)
     clocks.start()
     launches0 = m.launch_count()
-    ms_gen = timed(lambda: gen.run(hidden0, n_steps=n_dec), args.steps)
-    launches = m.launch_count() - launches0
+    ms_gen = timed(step_fn, args.steps)
+    launches = per_replay * args.steps if graph is not None else m.launch_count() - launches0
     clock_info = clocks.stop()
     assert m.device_status() == 0, "a bounded device wait gave up"
     value = aggregate_images_per_s(n_images, ms_gen, world)
@@ -364,8 +380,12 @@ def run_ours(args, cfg):
             "vs_baseline": None,
             "dtype": ("%s projections + bf16 attention/cache, fp32 accumulate" % ("fp16" if args.operand == "f16" else "bf16"))
                      if cfg.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": workload_config(cfg, ratio), "clocks": clock_info, "gpu_launches": int(launches),
-            "ms_per_decoding_step": ms_gen / cfg.T}
+            "config": dict(workload_config(cfg, ratio), launch=launch_mode), "clocks": clock_info,
+            "gpu_launches": int(launches), "ms_per_decoding_step": ms_gen / cfg.T}
+    if graph is not None and not args.no_extras:
+        ms_stream = timed(lambda: gen.run(hidden0), 2)
+        line["stream_launched"] = {"value": aggregate_images_per_s(n_images, ms_stream, world), "unit": "images/s",
+                                   "ms_per_step": ms_stream}
 
     if not args.no_extras:
         # ---- per-kernel-class device time of one more generation (an event in front of every
@@ -438,20 +458,6 @@ def run_ours(args, cfg):
             if dom["bound"] == "tensor":
                 line["roofline"]["frac_in_chain"] = line["kernels_in_chain"]["gemm_all"]["frac"]
                 line["roofline"]["achieved_in_chain"] = line["kernels_in_chain"]["gemm_all"]["achieved"]
-
-        # ---- the same generation captured once in a CUDA graph and replayed (no host launch cost at all)
-        if n_dec is None:
-            try:
-                l0 = m.launch_count()
-                graph = gen.capture(hidden0)
-                per_replay = (m.launch_count() - l0) // 2          # one eager generation, one recorded
-                graph.replay()
-                ms_graph = timed(lambda: graph.replay(), 2)
-                line["cuda_graph"] = {"value": world * n_images / (ms_graph * 1e-3), "unit": "images/s",
-                                      "ms_per_step": ms_graph, "kernel_nodes_per_replay": int(per_replay)}
-                assert m.device_status() == 0
-            except Exception as exc:                      # capture is an extra; the stream path is the benchmark
-                line["cuda_graph"] = {"unavailable": str(exc)[:200]}
 
         # ---- per-step latency: events between the steps of one more generation
         if n_dec is None:
@@ -697,6 +703,8 @@ def main():
                     help="stop each generation after this many decoding steps (profiling captures only)")
     ap.add_argument("--no-extras", action="store_true", help="only the timed region (for ncu launch lists)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--stream-launch", action="store_true",
+                    help="time the stream-launched generation instead of its CUDA-graph replay")
     ap.add_argument("--microbench", action="store_true",
                     help="Appendix-B style attention micro-benchmark instead of the generation benchmark")
     ap.add_argument("--operand", default="f16", choices=["f16", "bf16"],

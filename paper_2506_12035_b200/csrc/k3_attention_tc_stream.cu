@@ -130,6 +130,28 @@ MARCHE_DEVINL float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
 }
+// Packed fp32 pairs (one instruction for two values): (a0, a1) * m + (b, b), and pairwise accumulate.
+MARCHE_DEVINL void ffma2_bcast(float a0, float a1, float m, float b, float& r0, float& r1) {
+  asm("{\n"
+      ".reg .b64 ra, rm, rb, rr;\n"
+      "mov.b64 ra, {%2, %3};\n"
+      "mov.b64 rm, {%4, %4};\n"
+      "mov.b64 rb, {%5, %5};\n"
+      "fma.rn.f32x2 rr, ra, rm, rb;\n"
+      "mov.b64 {%0, %1}, rr;\n"
+      "}\n"
+      : "=f"(r0), "=f"(r1) : "f"(a0), "f"(a1), "f"(m), "f"(b));
+}
+MARCHE_DEVINL void fadd2(float& acc0, float& acc1, float p0, float p1) {
+  asm("{\n"
+      ".reg .b64 ra, rp;\n"
+      "mov.b64 ra, {%0, %1};\n"
+      "mov.b64 rp, {%2, %3};\n"
+      "add.f32x2 ra, ra, rp;\n"
+      "mov.b64 {%0, %1}, ra;\n"
+      "}\n"
+      : "+f"(acc0), "+f"(acc1) : "f"(p0), "f"(p1));
+}
 MARCHE_DEVINL float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -345,9 +367,10 @@ attention_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __
           if (lim >= KT) {                                 // (two copies of the loop: no per-element selects on the
 #pragma unroll                                             //  common, full tile)
             for (int c = 0; c < KT / 2; ++c) {
-              const float p0 = ex2_approx(fmaf(__uint_as_float(v[2 * c]), c_log2, neg));
-              const float p1 = ex2_approx(fmaf(__uint_as_float(v[2 * c + 1]), c_log2, neg));
-              ls[c & 3] += p0 + p1;
+              float x0, x1;
+              ffma2_bcast(__uint_as_float(v[2 * c]), __uint_as_float(v[2 * c + 1]), c_log2, neg, x0, x1);
+              const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+              fadd2(ls[2 * (c & 1)], ls[2 * (c & 1) + 1], p0, p1);
               v[c] = pack_bf16x2(p0, p1);
             }
           } else {
