@@ -54,27 +54,31 @@ def load_ncu_traffic():
     return out
 
 
-def write_ncu_traffic(csv_path):
-    """Reads `ncu -i <report> --page raw --csv` output and writes the mean DRAM bytes per launch of the
-    GEMM and attention kernels to profiles/ncu_dram_traffic.txt."""
+def write_ncu_traffic(csv_paths):
+    """Reads `ncu -i <report> --page raw --csv` outputs (comma-separated paths) and writes the mean DRAM
+    bytes per launch of the GEMM and attention kernels to profiles/ncu_dram_traffic.txt."""
     import csv
-    rows = list(csv.reader(open(csv_path)))
-    hdr = next(r for r in rows if "Kernel Name" in r)
-    units = rows[rows.index(hdr) + 1]
-    i_name = hdr.index("Kernel Name")
-    i_rd, i_wr = hdr.index("dram__bytes_read.sum"), hdr.index("dram__bytes_write.sum")
     scale = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
     acc = {}
-    for r in rows[rows.index(hdr) + 2:]:
-        if len(r) <= max(i_rd, i_wr):
-            continue
-        cls = "gemm" if "gemm_tcgen05" in r[i_name] else ("attention" if "attention" in r[i_name] else None)
-        if cls is None:
-            continue
-        b = float(r[i_rd].replace(",", "")) * scale[units[i_rd]] + float(r[i_wr].replace(",", "")) * scale[units[i_wr]]
-        acc.setdefault(cls, []).append(b)
+    for csv_path in csv_paths.split(","):
+        rows = list(csv.reader(open(csv_path)))
+        hdr = next(r for r in rows if "Kernel Name" in r)
+        units = rows[rows.index(hdr) + 1]
+        i_name = hdr.index("Kernel Name")
+        i_rd, i_wr = hdr.index("dram__bytes_read.sum"), hdr.index("dram__bytes_write.sum")
+        for r in rows[rows.index(hdr) + 2:]:
+            if len(r) <= max(i_rd, i_wr):
+                continue
+            name = r[i_name]
+            cls = "gemm" if "gemm_tcgen05" in name else ("attention" if "attention_mma" in name and ", 0>" in name else
+                                                         ("attention_tc_stream" if "attention_tc_stream" in name else None))
+            if cls is None:
+                continue
+            b = float(r[i_rd].replace(",", "")) * scale[units[i_rd]] + float(r[i_wr].replace(",", "")) * scale[units[i_wr]]
+            acc.setdefault(cls, []).append(b)
     with open(TRAFFIC_FILE, "w") as f:
-        f.write("# mean dram__bytes_read.sum + dram__bytes_write.sum per launch, from %s\n" % os.path.basename(csv_path))
+        f.write("# mean dram__bytes_read.sum + dram__bytes_write.sum per launch, from ncu --set full captures of\n"
+                "# 4-block slices of the benchmark workloads (see the *.md summaries beside this file for the commands)\n")
         f.write("# class bytes_per_launch launches\n")
         for cls, v in sorted(acc.items()):
             f.write("%s %.0f %d\n" % (cls, float(np.mean(v)), len(v)))

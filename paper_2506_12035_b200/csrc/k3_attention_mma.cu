@@ -84,6 +84,7 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap tmap_kv, const bf16* __
     // Fixed load sequence: per q-tile, [K tiles of the statistics pass,] then K+V tiles.
     if (lane == 0) {
       ptx::prefetch_tensormap(&tmap_kv);
+      const uint64_t stream_once = ptx::l2_policy_evict_first();
       int i = 0;
       for (; i < n_loads; ++i) {
         const int rem = i % (n_kv * PASSES);
@@ -93,8 +94,8 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap tmap_kv, const bf16* __
         if (!ptx::mbar_wait(empty_bar(s), ((uint32_t)(i / NSTAGE) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         const uint32_t dst = base + s * Cfg::STAGE_BYTES;
         ptx::mbar_expect_tx(full_bar(s), with_v ? Cfg::STAGE_BYTES : Cfg::TILE_BYTES);
-        ptx::tma_load_3d(dst, &tmap_kv, h * DH, kt * KT, b, full_bar(s));
-        if (with_v) ptx::tma_load_3d(dst + Cfg::TILE_BYTES, &tmap_kv, h * DH, kt * KT, B + b, full_bar(s));
+        ptx::tma_load_3d_hint(dst, &tmap_kv, h * DH, kt * KT, b, full_bar(s), stream_once);
+        if (with_v) ptx::tma_load_3d_hint(dst + Cfg::TILE_BYTES, &tmap_kv, h * DH, kt * KT, B + b, full_bar(s), stream_once);
       }
       if (!ok) {
         *(volatile int*)status = ST_ATTENTION;

@@ -224,6 +224,7 @@ attention_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __
       const int j = warp - W_PROD;
       ptx::prefetch_tensormap(&tmap_kv);
       ptx::prefetch_tensormap(&tmap_q);
+      const uint64_t stream_once = ptx::l2_policy_evict_first();
       int tl = 0;                                          // K/V tiles issued so far
       bool ok = true;
       for (int u = 0; u < n_units[j] && ok; ++u) {
@@ -236,8 +237,8 @@ attention_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __
           if (!ptx::mbar_wait(bar(j, B_KV_EMPTY + s), ((uint32_t)(tl / NST) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t dst = base + OFF_KV + (j * NST + s) * STAGE_BYTES;
           ptx::mbar_expect_tx(bar(j, B_KV_FULL + s), STAGE_BYTES);
-          ptx::tma_load_3d(dst, &tmap_kv, un.h * DH, kt * KT, un.b, bar(j, B_KV_FULL + s));
-          ptx::tma_load_3d(dst + K_BYTES, &tmap_kv, un.h * DH, kt * KT, B + un.b, bar(j, B_KV_FULL + s));
+          ptx::tma_load_3d_hint(dst, &tmap_kv, un.h * DH, kt * KT, un.b, bar(j, B_KV_FULL + s), stream_once);
+          ptx::tma_load_3d_hint(dst + K_BYTES, &tmap_kv, un.h * DH, kt * KT, B + un.b, bar(j, B_KV_FULL + s), stream_once);
         }
       }
       if (!ok) {

@@ -70,6 +70,20 @@ MARCHE_DEVINL void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
+// The same load with an L2 eviction-priority hint: data that is streamed once (the K/V cache during
+// attention) is marked evict-first so that it does not push the step's activations out of L2.
+MARCHE_DEVINL uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+MARCHE_DEVINL void tma_load_3d_hint(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar,
+                                    uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(policy)
+      : "memory");
+}
 // Bulk tensor stores from shared memory (row-major box, 128-byte swizzle), tracked by bulk groups.
 MARCHE_DEVINL void tma_store_2d(const CUtensorMap* map, int c0, int c1, uint32_t src) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
