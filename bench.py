@@ -517,9 +517,24 @@ def run_ours(args, cfg):
         gen.alloc_host_buffers(hidden0_np, rows_np, sets)
         for _ in range(2):
             h2d, d2h = gen.run_host()
-        ms_e2e = timed(lambda: gen.run_host(), args.steps)
+        e2e_fn, e2e_launch = (lambda: gen.run_host()), "stream launches"
+        if graph is not None:
+            # the same calls recorded once: the copies from / to the pinned host buffers become graph nodes
+            try:
+                side = torch.cuda.Stream()
+                g_e2e = torch.cuda.CUDAGraph()
+                with torch.cuda.stream(side):
+                    with torch.cuda.graph(g_e2e, stream=side):
+                        gen.run_host()
+                g_e2e.replay()
+                torch.cuda.synchronize()
+                e2e_fn, e2e_launch = (lambda: g_e2e.replay()), "one CUDA graph per generation, copies as graph nodes"
+            except Exception as exc:
+                e2e_launch = "stream launches (graph capture failed: %s)" % str(exc)[:120]
+        ms_e2e = timed(e2e_fn, args.steps)
         line["e2e"] = {"value": world * n_images / (ms_e2e * 1e-3), "unit": "images/s", "h2d_bytes_per_step": int(h2d),
-                       "d2h_bytes_per_step": int(d2h), "ms_per_step": ms_e2e}
+                       "d2h_bytes_per_step": int(d2h), "ms_per_step": ms_e2e, "launch": e2e_launch,
+                       "api": "marche_step_host: per step, inputs from pinned host memory, results back to it"}
         assert m.device_status() == 0
 
         # ---- CPU oracle on a bounded sample (rank 0, N = 1 only)
