@@ -365,6 +365,7 @@ attention_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __
           const float neg = -m_ref * c_log2;
           // weights: p = 2^((s - m_ref) / sqrt(d) * log2 e), packed bf16 pairs, in place (pair c -> v[c])
           float ls[4] = {0.f, 0.f, 0.f, 0.f};
+          bool half_stored = false;
           if (lim >= KT) {                                 // (two copies of the loop: no per-element selects on the
 #pragma unroll                                             //  common, full tile)
             for (int c = 0; c < KT / 2; ++c) {
@@ -373,7 +374,9 @@ attention_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __
               const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
               fadd2(ls[2 * (c & 1)], ls[2 * (c & 1) + 1], p0, p1);
               v[c] = pack_bf16x2(p0, p1);
+              if (c == KT / 4 - 1) tmem_st_32x16(t_p, v);  // first half on its way while the second is computed
             }
+            half_stored = true;
           } else {
 #pragma unroll
             for (int c = 0; c < KT / 2; ++c) {
@@ -386,7 +389,8 @@ attention_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __
             }
           }
           l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-          tmem_st_32x32(t_p, v);
+          if (half_stored) tmem_st_32x16(t_p + 16u, v + 16);
+          else tmem_st_32x32(t_p, v);
           tmem_st_wait();
         }
         ptx::tc_fence_before();

@@ -217,3 +217,36 @@ def test_context_is_bound_to_its_device():
     with torch.cuda.device(0):
         torch.cuda.synchronize()
         assert (out == -1).all()
+
+
+def test_measurement_hooks_change_launches_only_as_documented():
+    """marche_debug_repeat_classes / marche_debug_skip_classes: doubling the idempotent classes (LayerNorm, QKV
+    projection, attention, fc1) leaves the step's results bit-identical and adds exactly one launch per launch of
+    the class; leaving a class out removes its launches; other classes are refused."""
+    cfg = synth.CONFIGS["mar_b"].replace(L=2, E=0, B=8, T=6)
+    blocks = synth.make_weights(cfg)
+    m = make_model(cfg, blocks)
+    rng = np.random.default_rng(4)
+    hidden = dev(synth.make_hidden(cfg))
+    A = np.stack([rng.permutation(cfg.S)[:41] for _ in range(cfg.B)]).astype(np.int32)
+    G = A[:, :5]
+    n0 = m.launch_count()
+    out_ref, cache_ref, R_ref, _ = _one_step(m, cfg, hidden, A, G)
+    per_step = m.launch_count() - n0
+    idem = ["gather_layernorm", "gemm_qkv", "attention", "gemm_fc1_gelu"]
+    m.debug_repeat_classes(idem)
+    n0 = m.launch_count()
+    out_rep, cache_rep, R_rep, _ = _one_step(m, cfg, hidden, A, G)
+    assert m.launch_count() - n0 == per_step + 2 * cfg.L * 5           # two calls (full step, step): LN x2, qkv, attention, fc1
+    assert torch.equal(out_rep, out_ref) and torch.equal(cache_rep, cache_ref) and torch.equal(R_rep, R_ref)
+    m.debug_repeat_classes(())
+    m.debug_skip_classes(["attention"])
+    n0 = m.launch_count()
+    _one_step(m, cfg, hidden, A, G)
+    assert m.launch_count() - n0 == per_step - 2 * cfg.L
+    m.debug_skip_classes(())
+    with pytest.raises(MarcheError) as e:
+        m.debug_skip_classes(["topk"])
+    assert e.value.code == -1
+    out_again, _, _, _ = _one_step(m, cfg, hidden, A, G)
+    assert torch.equal(out_again, out_ref) and m.device_status() == 0
