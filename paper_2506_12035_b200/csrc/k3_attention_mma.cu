@@ -36,14 +36,30 @@ namespace {
 
 using namespace att;
 
+// Byte offset of 16-byte chunk c of key row r inside a K or V tile of this kernel.  head_dim 64: rows of 128
+// bytes under TMA's 128-byte swizzle.  head_dim 80: the tile arrives as two boxes, columns 0-63 (same layout)
+// and columns 64-79 behind them as rows of 32 bytes under the 32-byte swizzle, so that every ldmatrix phase
+// (8 rows x 16 bytes) touches all 32 banks once; packed 160-byte rows would make each phase a 2-way conflict,
+// and with two or three warps per CTA reading every tile that is what the kernel was bound by.
+// Ring depth: three 16 KB stages at head_dim 64; two 20 KB stages at head_dim 80, where a third would cost the
+// fourth resident CTA per SM.
+template <int DH> struct ring_stages { static constexpr int N = DH == 64 ? 3 : 2; };
+
+template <int DH> MARCHE_DEVINL uint32_t kv_off(int r, int c) {
+  if (DH == 64 || c < 8) return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4));
+  return (uint32_t)(KT * 128 + r * 32 + (((c - 8) ^ ((r >> 2) & 1)) << 4));
+}
+
 // NWARPS consumer warps (16 query rows each) plus one producer warp.
 template <int DH, int NWARPS, bool SCORING>
-__global__ void __launch_bounds__((NWARPS + 1) * 32, NWARPS == 3 ? 4 : 1)
-attention_mma_kernel(const __grid_constant__ CUtensorMap tmap_kv, const bf16* __restrict__ q, int ld_q, int n,
+__global__ void __launch_bounds__((NWARPS + 1) * 32, NWARPS == 3 ? 4 : ((NWARPS == 2 && DH == 80) ? 5 : 1))
+attention_mma_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_constant__ CUtensorMap tmap_tail,
+                     const bf16* __restrict__ q, int ld_q, int n,
                      int S, int H, int B, const uint8_t* __restrict__ is_new, float* __restrict__ score_partial,
                      uint16_t* __restrict__ o, bool o_bf16, int* __restrict__ status) {
   using Cfg = AttCfg<DH>;
   constexpr int QT = NWARPS * 16;
+  constexpr int NSTAGE = ring_stages<DH>::N;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -96,6 +112,12 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap tmap_kv, const bf16* __
         ptx::mbar_expect_tx(full_bar(s), with_v ? Cfg::STAGE_BYTES : Cfg::TILE_BYTES);
         ptx::tma_load_3d_hint(dst, &tmap_kv, h * DH, kt * KT, b, full_bar(s), stream_once);
         if (with_v) ptx::tma_load_3d_hint(dst + Cfg::TILE_BYTES, &tmap_kv, h * DH, kt * KT, B + b, full_bar(s), stream_once);
+        if (DH > 64) {                                     // columns 64 .. DH-1 as a second box behind the first
+          ptx::tma_load_3d_hint(dst + KT * 128, &tmap_tail, h * DH + 64, kt * KT, b, full_bar(s), stream_once);
+          if (with_v)
+            ptx::tma_load_3d_hint(dst + Cfg::TILE_BYTES + KT * 128, &tmap_tail, h * DH + 64, kt * KT, B + b, full_bar(s),
+                                  stream_once);
+        }
       }
       if (!ok) {
         *(volatile int*)status = ST_ATTENTION;
@@ -162,7 +184,7 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap tmap_kv, const bf16* __
             const int mi = lane >> 3;
             const int key = 8 * (2 * jp + (mi >> 1)) + (lane & 7);
             uint32_t b0, b1, b2, b3;
-            ldsm_x4(k_tile + tile_off<DH>(key, 2 * kk + (mi & 1)), b0, b1, b2, b3);
+            ldsm_x4(k_tile + kv_off<DH>(key, 2 * kk + (mi & 1)), b0, b1, b2, b3);
             mma_bf16(sacc[2 * jp], qf[kk], b0, b1);
             mma_bf16(sacc[2 * jp + 1], qf[kk], b2, b3);
           }
@@ -261,7 +283,7 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap tmap_kv, const bf16* __
               const int mi = lane >> 3;
               const int key = 16 * k2 + 8 * (mi & 1) + (lane & 7);
               uint32_t b0, b1, b2, b3;
-              ldsm_x4_trans(v_tile + tile_off<DH>(key, jd + (mi >> 1)), b0, b1, b2, b3);
+              ldsm_x4_trans(v_tile + kv_off<DH>(key, jd + (mi >> 1)), b0, b1, b2, b3);
               mma_bf16(oacc[jd], pf, b0, b1);
               mma_bf16(oacc[jd + 1], pf, b2, b3);
             }
@@ -303,28 +325,29 @@ attention_mma_kernel(const __grid_constant__ CUtensorMap tmap_kv, const bf16* __
 }
 
 template <int DH, int NWARPS, bool SCORING>
-cudaError_t launch_att(const CUtensorMap& tm, const bf16* q, int ld_q, int B, int n, int S, int H,
+cudaError_t launch_att(const CUtensorMap& tm, const CUtensorMap& tail, const bf16* q, int ld_q, int B, int n, int S, int H,
                        const uint8_t* is_new, float* partial, uint16_t* o, bool o_bf16, int* status, cudaStream_t st) {
+  constexpr int NSTAGE = ring_stages<DH>::N;
   const size_t smem = NSTAGE * AttCfg<DH>::STAGE_BYTES + 1024 + 64 + (SCORING ? (size_t)NWARPS * S * sizeof(float) : 0);
   static size_t smem_set[kMaxDevices] = {};
   cudaError_t e = ensure_dynamic_smem(attention_mma_kernel<DH, NWARPS, SCORING>, smem, smem_set);
   if (e != cudaSuccess) return e;
   // (Launching one sample's heads as a cluster, to co-schedule the CTAs that read neighbouring
   // 128-byte pieces of the same cache rows, was measured and does not help: 41.0 -> 41-43 us.)
-  return launch_pdl(attention_mma_kernel<DH, NWARPS, SCORING>, dim3(B * H), dim3((NWARPS + 1) * 32), smem, st, tm, q, ld_q,
+  return launch_pdl(attention_mma_kernel<DH, NWARPS, SCORING>, dim3(B * H), dim3((NWARPS + 1) * 32), smem, st, tm, tail, q, ld_q,
                     n, S, H, B, is_new, partial, o, o_bf16, status);
 }
 
 template <int DH>
-cudaError_t launch_dh(const CUtensorMap& tm, const bf16* q, int ld_q, int B, int n, int S, int H,
+cudaError_t launch_dh(const CUtensorMap& tm, const CUtensorMap& tail, const bf16* q, int ld_q, int B, int n, int S, int H,
                       const uint8_t* is_new, float* partial, uint16_t* o, bool o_bf16, int* status, cudaStream_t st) {
   const bool sc = is_new != nullptr;
   // 7 consumer warps + the producer warp = 256 threads: two CTAs per SM still fit the register file
   const int nw = n <= 16 ? 1 : (n <= 32 ? 2 : (n <= 48 ? 3 : (n <= 64 ? 4 : 7)));
 #define MARCHE_ATT_CASE(NW_)                                                                              \
   if (nw == NW_)                                                                                          \
-    return sc ? launch_att<DH, NW_, true>(tm, q, ld_q, B, n, S, H, is_new, partial, o, o_bf16, status, st) \
-              : launch_att<DH, NW_, false>(tm, q, ld_q, B, n, S, H, is_new, partial, o, o_bf16, status, st);
+    return sc ? launch_att<DH, NW_, true>(tm, tail, q, ld_q, B, n, S, H, is_new, partial, o, o_bf16, status, st) \
+              : launch_att<DH, NW_, false>(tm, tail, q, ld_q, B, n, S, H, is_new, partial, o, o_bf16, status, st);
   MARCHE_ATT_CASE(1) MARCHE_ATT_CASE(2) MARCHE_ATT_CASE(3) MARCHE_ATT_CASE(4) MARCHE_ATT_CASE(7)
 #undef MARCHE_ATT_CASE
   return cudaErrorInvalidValue;
@@ -342,11 +365,14 @@ cudaError_t launch_attention_mma(const void* q, int ld_q, int B, int n, int S, i
   CUtensorMap tm;
   const uint64_t dims[3] = {(uint64_t)D, (uint64_t)S, (uint64_t)2 * B};
   const uint64_t strides[2] = {(uint64_t)D * 2, (uint64_t)S * D * 2};
-  const uint32_t box[3] = {(uint32_t)dh, KT, 1};
-  if (!tma_make_map_bf16(&tm, cache_layer, 3, dims, strides, box, dh == 64)) return cudaErrorInvalidValue;
+  const uint32_t box[3] = {64, KT, 1};                   // columns 0-63 of a head: 128-byte rows, swizzled
+  if (!tma_make_map_bf16(&tm, cache_layer, 3, dims, strides, box, true)) return cudaErrorInvalidValue;
   if (dh == 64)
-    return launch_dh<64>(tm, (const bf16*)q, ld_q, B, n, S, H, is_new, score_partial, (uint16_t*)o, o_bf16, status, st);
-  return launch_dh<80>(tm, (const bf16*)q, ld_q, B, n, S, H, is_new, score_partial, (uint16_t*)o, o_bf16, status, st);
+    return launch_dh<64>(tm, tm, (const bf16*)q, ld_q, B, n, S, H, is_new, score_partial, (uint16_t*)o, o_bf16, status, st);
+  CUtensorMap tail;                                      // columns 64-79: 32-byte rows, 32-byte swizzle
+  const uint32_t box_tail[3] = {16, KT, 1};
+  if (!tma_make_map_bf16(&tail, cache_layer, 3, dims, strides, box_tail, false, false, true)) return cudaErrorInvalidValue;
+  return launch_dh<80>(tm, tail, (const bf16*)q, ld_q, B, n, S, H, is_new, score_partial, (uint16_t*)o, o_bf16, status, st);
 }
 
 }  // namespace marche

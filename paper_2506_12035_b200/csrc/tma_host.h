@@ -28,10 +28,12 @@ inline EncodeTiledFn tma_encode_fn() {
 }
 
 // 16-bit (bf16, or fp16 when ieee_half) tensor of `rank` dimensions (innermost first).  strides_bytes has rank-1 entries
-// (the innermost stride is the element size).  Out-of-bounds elements read as zero.
+// (the innermost stride is the element size).  Out-of-bounds elements read as zero.  swizzle128 / swizzle32: the
+// box's rows are 128 / 32 bytes wide and their 16-byte chunks are permuted in shared memory (bank-conflict-free
+// ldmatrix); neither: rows packed as they are.
 inline bool tma_make_map_bf16(CUtensorMap* map, const void* ptr, int rank, const uint64_t* dims,
                               const uint64_t* strides_bytes, const uint32_t* box, bool swizzle128,
-                              bool ieee_half = false) {
+                              bool ieee_half = false, bool swizzle32 = false) {
   EncodeTiledFn fn = tma_encode_fn();
   if (!fn) return false;
   cuuint64_t d[5], s[5];
@@ -44,7 +46,8 @@ inline bool tma_make_map_bf16(CUtensorMap* map, const void* ptr, int rank, const
   }
   return fn(map, ieee_half ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank,
             const_cast<void*>(ptr), d, s, b, e,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+            CU_TENSOR_MAP_INTERLEAVE_NONE,
+            swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : (swizzle32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE),
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
