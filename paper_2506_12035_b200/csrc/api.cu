@@ -238,6 +238,11 @@ int do_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void* ca
   else if (tc5)
     MARCHE_TRY(launch_attention_tcgen05(q, ld_q, c.batch, n, S, c.n_heads, c.head_dim, cache_layer, is_new,
                                         partial, o, ctx->a_bf16, ctx->status_dev, st), "attention_tcgen05");
+  else if (!is_new && n <= 32 && ld_q % 8 == 0 && ((uintptr_t)q & 15) == 0)
+    // very small active sets, no scores: the persistent launch of the same arithmetic (31 vs 34 us at n = 8,
+    // 32 vs 36 us at n = 24..32, S 320); above 32 rows one CTA per item is as fast or faster
+    MARCHE_TRY(launch_attention_mma_persist(q, ld_q, c.batch, n, S, c.n_heads, c.head_dim, cache_layer, o, ctx->a_bf16,
+                                            ctx->status_dev, st), "attention_mma_persist");
   else
     MARCHE_TRY(launch_attention_mma(q, ld_q, c.batch, n, S, c.n_heads, c.head_dim, cache_layer, is_new,
                                     partial, o, ctx->a_bf16, ctx->status_dev, st), "attention_mma");

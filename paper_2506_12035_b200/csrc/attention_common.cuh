@@ -41,6 +41,20 @@ template <int DH> MARCHE_DEVINL uint32_t tile_off(int r, int c) {
   return (uint32_t)(r * AttCfg<DH>::ROWB + (c << 4));
 }
 
+// Ring depth of the mma.sync kernels (plain and persistent): three 16 KB stages at head_dim 64; two 20 KB stages
+// at head_dim 80, where a third would cost the fourth resident CTA per SM.
+template <int DH> struct ring_stages { static constexpr int N = DH == 64 ? 3 : 2; };
+
+// Byte offset of 16-byte chunk c of key row r inside a K or V tile of those kernels.  head_dim 64: rows of 128
+// bytes under TMA's 128-byte swizzle.  head_dim 80: the tile arrives as two boxes, columns 0-63 (same layout)
+// and columns 64-79 behind them as rows of 32 bytes under the 32-byte swizzle, so that every ldmatrix phase
+// (8 rows x 16 bytes) touches all 32 banks once; packed 160-byte rows would make each phase a 2-way conflict,
+// and with two or three warps per CTA reading every tile that is what the kernel was bound by.
+template <int DH> MARCHE_DEVINL uint32_t kv_off(int r, int c) {
+  if (DH == 64 || c < 8) return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4));
+  return (uint32_t)(KT * 128 + r * 32 + (((c - 8) ^ ((r >> 2) & 1)) << 4));
+}
+
 MARCHE_DEVINL float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));

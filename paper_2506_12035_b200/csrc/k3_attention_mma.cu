@@ -36,20 +36,6 @@ namespace {
 
 using namespace att;
 
-// Byte offset of 16-byte chunk c of key row r inside a K or V tile of this kernel.  head_dim 64: rows of 128
-// bytes under TMA's 128-byte swizzle.  head_dim 80: the tile arrives as two boxes, columns 0-63 (same layout)
-// and columns 64-79 behind them as rows of 32 bytes under the 32-byte swizzle, so that every ldmatrix phase
-// (8 rows x 16 bytes) touches all 32 banks once; packed 160-byte rows would make each phase a 2-way conflict,
-// and with two or three warps per CTA reading every tile that is what the kernel was bound by.
-// Ring depth: three 16 KB stages at head_dim 64; two 20 KB stages at head_dim 80, where a third would cost the
-// fourth resident CTA per SM.
-template <int DH> struct ring_stages { static constexpr int N = DH == 64 ? 3 : 2; };
-
-template <int DH> MARCHE_DEVINL uint32_t kv_off(int r, int c) {
-  if (DH == 64 || c < 8) return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4));
-  return (uint32_t)(KT * 128 + r * 32 + (((c - 8) ^ ((r >> 2) & 1)) << 4));
-}
-
 // NWARPS consumer warps (16 query rows each) plus one producer warp.
 template <int DH, int NWARPS, bool SCORING>
 __global__ void __launch_bounds__((NWARPS + 1) * 32, NWARPS == 3 ? 4 : ((NWARPS == 2 && DH == 80) ? 5 : 1))

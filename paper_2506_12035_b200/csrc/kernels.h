@@ -103,6 +103,11 @@ cudaError_t launch_attention_mma(const void* q, int ld_q, int B, int n, int S, i
                                  const void* cache_layer, const uint8_t* is_new, float* score_partial, void* o,
                                  bool o_bf16, int* status, cudaStream_t st);
 
+// The same kernel's plain flavour for n <= 32 as a persistent launch (equal item shares per resident CTA, loads
+// running ahead across items, query rows by TMA).  ld_q % 8 == 0; q and cache_layer 16-byte aligned.
+cudaError_t launch_attention_mma_persist(const void* q, int ld_q, int B, int n, int S, int H, int dh,
+                                         const void* cache_layer, void* o, bool o_bf16, int* status, cudaStream_t st);
+
 // K3 on tcgen05 (head_dim 64 only): S = Q K^T and O = P V as tcgen05.mma with TMEM accumulators.
 // ld_q % 8 == 0; q and cache_layer 16-byte aligned.
 cudaError_t launch_attention_tcgen05(const void* q, int ld_q, int B, int n, int S, int H, int dh,

@@ -440,6 +440,39 @@ def test_attention_many_rows(S, dh, H, n, nG):
 
 
 @pytest.mark.parametrize("operand", ["bf16", "bf16b"])
+@pytest.mark.parametrize("dh", [64, 80])
+@pytest.mark.parametrize("B,H,S,n", [(2, 4, 68, 1), (3, 4, 257, 7), (2, 8, 320, 16), (2, 8, 320, 17), (5, 4, 64, 32),
+                                     (80, 16, 200, 5), (140, 8, 130, 20)])
+def test_attention_small_sets_persistent(operand, dh, B, H, S, n):
+    """Plain attention at up to 32 query rows takes the persistent mma.sync launch: one and two consumer warps,
+    both head sizes, ragged key tiles, fewer items than resident CTAs and several items per CTA (1280 and 1120
+    items), where a CTA's loads run ahead into its next item."""
+    if dh == 80:
+        H = (H + 7) // 8 * 8                                # the model width must be a multiple of 128
+    D = H * dh
+    if operand == "bf16b" and B > 5:
+        pytest.skip("one operand type is enough for the large shapes")
+    cfg, blocks, m = model_for(operand, D, H, 128, S, B)
+    rng = np.random.default_rng(7 * B + H + S + n + dh)
+    cache = rng.standard_normal((2, B, S, D)).astype(np.float32)
+    q = (rng.standard_normal((B * n, D)) * 2.0).astype(np.float32)
+    o = torch.zeros(B * n, D, dtype=adt(operand), device="cuda")
+    m.attention(dev(q, torch.bfloat16), D, n, dev(cache, torch.bfloat16), None, None, o)
+    torch.cuda.synchronize()
+    assert m.device_status() == 0
+    got = host(o).reshape(B, n, D)
+    assert np.isfinite(got).all()
+    qq, cc = quant(q, "bf16").reshape(B, n, D), quant(cache, "bf16")
+    for b in sorted(set([0, 1, B // 2, B - 2, B - 1])):
+        want = np.zeros((n, D))
+        for h in range(H):
+            c = slice(h * dh, (h + 1) * dh)
+            want[:, c], _ = orc.softmax_attention(qq[b][:, c], cc[0, b][:, c], cc[1, b][:, c])
+        assert rel_l2(got[b], want) <= 8e-3 and max_abs(got[b], want) <= 3e-2, \
+            "b=%d: max-abs %.3g rel-L2 %.3g" % (b, max_abs(got[b], want), rel_l2(got[b], want))
+
+
+@pytest.mark.parametrize("operand", ["bf16", "bf16b"])
 @pytest.mark.parametrize("B,H,S,n", [(2, 4, 68, 5), (2, 4, 128, 128), (3, 4, 320, 41), (40, 4, 320, 41), (2, 4, 320, 129),
                                      (2, 4, 320, 320), (100, 4, 320, 77), (2, 16, 1088, 122), (2, 16, 1088, 159),
                                      (1, 4, 1088, 1088), (2, 4, 2048, 300), (37, 8, 300, 257)])
