@@ -53,8 +53,7 @@ MARCHE_DEVINL void epilogue_box(uint32_t t_addr, const float* __restrict__ bias_
         float v4 = __uint_as_float(r[8 * j + 4]) + b1.x, v5 = __uint_as_float(r[8 * j + 5]) + b1.y;
         float v6 = __uint_as_float(r[8 * j + 6]) + b1.z, v7 = __uint_as_float(r[8 * j + 7]) + b1.w;
         if (EPI == 2) {
-          v0 = gelu_erf_fast(v0); v1 = gelu_erf_fast(v1); v2 = gelu_erf_fast(v2); v3 = gelu_erf_fast(v3);
-          v4 = gelu_erf_fast(v4); v5 = gelu_erf_fast(v5); v6 = gelu_erf_fast(v6); v7 = gelu_erf_fast(v7);
+          gelu_erf_pair(v0, v1); gelu_erf_pair(v2, v3); gelu_erf_pair(v4, v5); gelu_erf_pair(v6, v7);
         }
         const uint32_t dst = row_base + (uint32_t)(((hh * 4 + j) ^ (lane & 7)) << 4);
         uint32_t p0, p1, p2, p3;
