@@ -453,7 +453,7 @@ typedef struct {
   int32_t stream_k;              /* 1: fc2-sized residual projections use stream-K with ordered reduce-adds   */
   int32_t fuse_qkv_scatter;      /* 1: the QKV projection's epilogue writes K, V into the cache (no K5 launch)*/
   int32_t attention_kernel;      /* MARCHE_ATTENTION_*: AUTO picks by active rows and head_dim                 */
-  int32_t attention_tc_min_rows; /* AUTO: tcgen05 attention above this many active rows (head_dim 64; 60)      */
+  int32_t attention_tc_min_rows; /* AUTO: tcgen05 attention above this many active rows (head_dim 64; 48)      */
   int32_t two_segment_attention; /* 1: the step uses marche_attention_two_segment instead of K5 + K3           */
   int32_t gemm_kernel;           /* MARCHE_GEMM_*: AUTO = CTA-pair kernel above 128 rows                       */
   int32_t tail_split;            /* 0 off, 1 cost model, 2 / 4 forced: column slices in a partial last round   */

@@ -112,7 +112,7 @@ marche_tuning default_tuning() {
   t.stream_k = 1;
   t.fuse_qkv_scatter = 1;
   t.attention_kernel = MARCHE_ATTENTION_AUTO;
-  t.attention_tc_min_rows = 60;
+  t.attention_tc_min_rows = 48;
   t.two_segment_attention = 0;
   t.gemm_kernel = MARCHE_GEMM_AUTO;
   t.tail_split = 1;
@@ -221,9 +221,10 @@ int do_attention(marche_ctx* ctx, const void* q, int ld_q, int n, const void* ca
   for (int rep_i = 0; rep_i < launches_of(ctx, MARCHE_KC_ATTENTION); ++rep_i) {
   if (n > 0) mark(ctx, MARCHE_KC_ATTENTION, st);
   // Three tensor-core kernels.  At small active sets the step is bound by streaming the cache and the
-  // mma.sync kernel (several small CTAs per SM, one pass) is fastest: 43 us vs 51 us at n = 41 (S 320).
-  // From about 60 rows the single-pass tcgen05 kernel wins (S 320: 53 vs 58 us at n = 64, 54 vs 110 us at
-  // n = 77, 151 vs 303 us at n = 320; S 1088: 83 vs 252 us at n = 116, 137 vs 256 us at n = 159).  The
+  // mma.sync kernel (several small CTAs per SM, one pass) is fastest: 40 us vs 50 us at n = 41..48 (S 320).
+  // From 49 rows, where the mma.sync kernel needs a fourth consumer warp and drops to two CTAs per SM, the
+  // single-pass tcgen05 kernel wins (S 320: 50 vs 56 us at n = 49..64, 54 vs 110 us at n = 77, 141 vs 303 us at
+  // n = 320; S 1088: 77 vs 82 us at n = 49..64, 81 vs 252 us at n = 116, 129 vs 256 us at n = 159).  The
   // relevance scores need final weights, hence the two-pass tcgen05 kernel there (74 vs 143 us at n = 77).
   // marche_tuning.attention_kernel forces one of them; head_dim 80 has only the mma.sync kernel.
   const int tc_min = is_new ? 64 : ctx->tune.attention_tc_min_rows;

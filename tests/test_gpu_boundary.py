@@ -78,7 +78,7 @@ def test_tuning_alternatives_compute_the_same_step():
     blocks = synth.make_weights(cfg)
     m = make_model(cfg, blocks)
     defaults = m.get_tuning()
-    assert defaults == dict(stream_k=1, fuse_qkv_scatter=1, attention_kernel=0, attention_tc_min_rows=60,
+    assert defaults == dict(stream_k=1, fuse_qkv_scatter=1, attention_kernel=0, attention_tc_min_rows=48,
                             two_segment_attention=0, gemm_kernel=0, tail_split=1, tile_n=0, pdl=1)
     rng = np.random.default_rng(1)
     hidden_np = synth.make_hidden(cfg)
