@@ -66,18 +66,18 @@ MARCHE_DEVINL float warp_max(float v) {
 MARCHE_DEVINL float gelu_erf(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752440f)); }
 
 // GELU of two values at once for the tensor-core epilogue, without the special-function unit (which, at a
-// quarter of the FP32 rate, was what the fc1 epilogue waited for): erf(x / sqrt 2) = x R(x^2) on |x| <= 3 sqrt 2
-// with R a degree-8 polynomial (fitted to erf, absolute error <= 2.3e-5 including the clamp at erf(3) = 1 - 2.2e-5),
-// evaluated for both values with packed fp32-pair instructions; GELU = 0.5 x + 0.5 x erf.  The error in the
-// result, <= 1.2e-5 |x|, is a tenth of the 16-bit rounding it is followed by.
+// quarter of the FP32 rate, was what the fc1 epilogue waited for): GELU(x) = x Phi(x) with
+// Phi(x) = sat(0.5 + x R(x^2)), R a degree-8 polynomial fitted to erf(x / sqrt 2) / (2 x) on |x| <= 3 sqrt 2.
+// Beyond that range x R(x^2) keeps growing in magnitude (positive leading coefficient, checked numerically: it
+// never comes back below 0.49999), so the saturating FMA clamps Phi to 0 or 1 there, infinities included.  The
+// polynomial runs for both values in packed fp32-pair instructions.  Error: <= 1.2e-5 in Phi, <= 4.8e-5 absolute
+// in the result, a tenth of the 16-bit rounding it is followed by.
 MARCHE_DEVINL void gelu_erf_pair(float& a, float& b) {
-  const float c = 4.2426405f;
-  const float ac = fminf(fmaxf(a, -c), c), bc = fminf(fmaxf(b, -c), c);
+  float ra, rb;
   asm("{\n"
-      ".reg .b64 x, xc, u, acc, k, h;\n"
-      "mov.b64 x, {%0, %1};\n"
-      "mov.b64 xc, {%2, %3};\n"
-      "mul.f32x2 u, xc, xc;\n"
+      ".reg .b64 x, u, acc, k;\n"
+      "mov.b64 x, {%2, %3};\n"
+      "mul.f32x2 u, x, x;\n"
       "mov.b64 acc, {%4, %4};\n"
       "mov.b64 k, {%5, %5};\n fma.rn.f32x2 acc, acc, u, k;\n"
       "mov.b64 k, {%6, %6};\n fma.rn.f32x2 acc, acc, u, k;\n"
@@ -87,15 +87,17 @@ MARCHE_DEVINL void gelu_erf_pair(float& a, float& b) {
       "mov.b64 k, {%10, %10};\n fma.rn.f32x2 acc, acc, u, k;\n"
       "mov.b64 k, {%11, %11};\n fma.rn.f32x2 acc, acc, u, k;\n"
       "mov.b64 k, {%12, %12};\n fma.rn.f32x2 acc, acc, u, k;\n"
-      "mul.f32x2 acc, acc, xc;\n"                       // erf
-      "mov.b64 k, {%13, %13};\n mul.f32x2 h, x, k;\n"   // x / 2
-      "fma.rn.f32x2 x, h, acc, h;\n"
-      "mov.b64 {%0, %1}, x;\n"
+      "mov.b64 {%0, %1}, acc;\n"
       "}\n"
-      : "+f"(a), "+f"(b)
-      : "f"(ac), "f"(bc), "f"(1.125353213e-10f), "f"(-1.074373479e-08f), "f"(4.536591405e-07f), "f"(-1.129242810e-05f),
-        "f"(1.871812274e-04f), "f"(-2.218800364e-03f), "f"(1.963623799e-02f), "f"(-1.326938421e-01f),
-        "f"(7.978062630e-01f), "f"(0.5f));
+      : "=f"(ra), "=f"(rb)
+      : "f"(a), "f"(b), "f"(0.5f * 1.125353213e-10f), "f"(0.5f * -1.074373479e-08f), "f"(0.5f * 4.536591405e-07f),
+        "f"(0.5f * -1.129242810e-05f), "f"(0.5f * 1.871812274e-04f), "f"(0.5f * -2.218800364e-03f),
+        "f"(0.5f * 1.963623799e-02f), "f"(0.5f * -1.326938421e-01f), "f"(0.5f * 7.978062630e-01f));
+  float pa, pb;
+  asm("fma.rn.sat.f32 %0, %1, %2, 0f3F000000;" : "=f"(pa) : "f"(a), "f"(ra));
+  asm("fma.rn.sat.f32 %0, %1, %2, 0f3F000000;" : "=f"(pb) : "f"(b), "f"(rb));
+  a *= pa;
+  b *= pb;
 }
 
 // Stores 4 consecutive outputs of type T starting at a 4-element aligned column.
