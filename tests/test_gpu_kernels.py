@@ -108,6 +108,37 @@ def test_linear_all_epilogues(dtype, M, N, K):
     assert max_abs(host(out), want) <= (3e-2 if dtype in LOW else 1e-4)
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "bf16b"])
+def test_gelu_epilogue_over_the_whole_input_range(dtype):
+    """The GELU of the tensor-core epilogue (a polynomial for erf, saturating beyond |x| = 3 sqrt 2) against the
+    oracle's erf GELU on a dense grid: a selection matrix as the weight and the grid as bias make the accumulator
+    equal the grid value exactly, so the only differences are the approximation and the 16-bit rounding of the
+    result.  Grid: -12 .. 12 in steps of 1/512 (covers the fitted range, the clamp point and the saturated tails),
+    plus large magnitudes up to the fp16 maximum."""
+    cfg, blocks, m = model_for(dtype, 256, 4, 1024, 68, 2)
+    M, N, K = 128, 12288 + 128, 64
+    grid = np.concatenate([np.arange(-12.0, 12.0, 1.0 / 512.0),
+                           np.array([-65000.0, -1000.0, -100.0, -13.0, 13.0, 100.0, 1000.0, 60000.0]),
+                           np.zeros(120)]).astype(np.float32)
+    assert grid.shape[0] == N
+    a = np.zeros((M, K), np.float32)                                    # accumulator = bias exactly
+    w = np.zeros((N, K), np.float32)
+    out = torch.zeros(M, N, dtype=adt(dtype), device="cuda")
+    m.linear(dev(a, adt(dtype)), dev(w, adt(dtype)), dev(grid), 2, out)
+    torch.cuda.synchronize()
+    got = host(out)
+    assert (got == got[0:1]).all()                                      # every row the same function of the bias
+    want = orc.gelu(grid.astype(np.float64))
+    if dtype == "bf16":                                                 # fp16 result: saturates at 65504
+        want = np.clip(want, -65504.0, 65504.0)
+    eps = 2.0 ** -11 if dtype == "bf16" else 2.0 ** -8                  # half an ulp, relative
+    err = np.abs(got[0] - want)
+    bound = eps * np.abs(want) + 1.0e-4                                 # rounding + the approximation (<= 4.8e-5)
+    worst = int(np.argmax(err - bound))
+    assert (err <= bound).all(), "x = %g: got %g, want %g" % (grid[worst], got[0][worst], want[worst])
+    assert (got[0][grid <= -13.0] == 0).all() and np.isfinite(got).all()
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16", "bf16b"])
 def test_linear_strided_input_and_row_guard(dtype):
     """a is a column slice of a wider matrix (lda > K); rows >= M of `out` stay untouched."""
